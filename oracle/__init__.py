@@ -1,0 +1,114 @@
+"""ctypes front end of the CPU oracle (`nsd_oracle.cpp`).
+
+TEST INFRASTRUCTURE, NOT PRODUCT: only `tests/`, the smoke check and the
+benchmark's cpu_baseline / reference arm may import this package.  It neither
+imports nor is imported by the CUDA package.  Arrays are numpy, on the host;
+bf16 tensors travel as uint16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "nsd_oracle.cpp")
+_SO = os.path.join(_HERE, "libnsd_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no CUDA involved). Returns the .so path."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-pthread", "-ffp-contract=off",
+               "-o", _SO, _SRC]
+        subprocess.run(cmd, check=True)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i32, i64, vp = ctypes.c_int, ctypes.c_int64, ctypes.c_void_p
+        lib.oracle_hardware_threads.restype = i32
+        lib.oracle_kv_prepare.restype = i32
+        lib.oracle_kv_prepare.argtypes = [vp, i32, i64, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i32, i32]
+        lib.oracle_verify_attn.restype = i32
+        lib.oracle_verify_attn.argtypes = [vp, i32, i64, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, i32, vp, i32, i32]
+        lib.oracle_spec_accept.restype = i32
+        lib.oracle_spec_accept.argtypes = [vp, vp, vp, vp, vp, i32, i32, i64, vp, vp, vp, vp, i32]
+        _lib = lib
+    return _lib
+
+
+def hardware_threads() -> int:
+    return int(_load().oracle_hardware_threads())
+
+
+def _ptr(a: Optional[np.ndarray], dtype) -> Optional[int]:
+    if a is None:
+        return None
+    assert isinstance(a, np.ndarray) and a.dtype == dtype and a.flags["C_CONTIGUOUS"], (a.dtype, dtype)
+    return a.ctypes.data
+
+
+def kv_prepare(pool, mig_indptr, mig_src, mig_dst, ctx_len, kv_indptr, kv_indices, k_new, v_new,
+               gamma: int, layer_begin: int = 0, layer_count: Optional[int] = None) -> int:
+    """In place on `pool` (uint16 [num_slabs][num_blocks][2][Hkv][bs][D]).
+
+    `k_new`/`v_new`: uint16 [num_layers][batch*(gamma+1)][Hkv][D] or None (no append).
+    """
+    S, NB, two, Hkv, bs, D = pool.shape
+    assert two == 2
+    n_mig = len(mig_indptr) - 1 if mig_indptr is not None else 0
+    batch = len(ctx_len)
+    if layer_count is None:
+        layer_count = (k_new.shape[0] if k_new is not None else S) - layer_begin
+    if k_new is not None:
+        assert k_new.shape[1:] == (batch * (gamma + 1), Hkv, D) and v_new.shape == k_new.shape
+    return _load().oracle_kv_prepare(
+        _ptr(pool, np.uint16), S, NB, Hkv, bs, D, n_mig, _ptr(mig_indptr, np.int64), _ptr(mig_src, np.int32),
+        _ptr(mig_dst, np.int32), batch, gamma, _ptr(ctx_len, np.int32), _ptr(kv_indptr, np.int64),
+        _ptr(kv_indices, np.int32), _ptr(k_new, np.uint16), _ptr(v_new, np.uint16), layer_begin, layer_count)
+
+
+def verify_attn(pool, q, ctx_len, kv_indptr, kv_indices, gamma: int, layer: int = 0,
+                req_list: Optional[np.ndarray] = None, want_lse: bool = False, nthreads: Optional[int] = None):
+    """Returns o fp32 [rows][Hq][D] (and lse [rows][Hq] when asked).  Rows of
+    requests outside `req_list` are left as NaN."""
+    S, NB, two, Hkv, bs, D = pool.shape
+    rows, Hq, D2 = q.shape
+    batch = len(ctx_len)
+    assert D2 == D and rows == batch * (gamma + 1)
+    o = np.full((rows, Hq, D), np.nan, dtype=np.float32)
+    lse = np.full((rows, Hq), np.nan, dtype=np.float32) if want_lse else None
+    nt = nthreads or hardware_threads()
+    rc = _load().oracle_verify_attn(
+        _ptr(pool, np.uint16), S, NB, Hq, Hkv, bs, D, _ptr(q, np.uint16), _ptr(o, np.float32),
+        _ptr(lse, np.float32), batch, gamma, _ptr(ctx_len, np.int32), _ptr(kv_indptr, np.int64),
+        _ptr(kv_indices, np.int32), layer, _ptr(req_list, np.int32), 0 if req_list is None else len(req_list), nt)
+    if rc != 0:
+        raise RuntimeError(f"oracle_verify_attn failed: {rc}")
+    return (o, lse) if want_lse else o
+
+
+def spec_accept(p, q, draft_tok, u_acc, u_smp, ctx_len: Optional[np.ndarray] = None, nthreads: Optional[int] = None):
+    """Returns (acc_len [B], out_tok [B][gamma+1], new_ctx_len [B] or None)."""
+    B, g1, V = p.shape
+    gamma = g1 - 1
+    assert q.shape == (B, gamma, V) and draft_tok.shape == (B, gamma) and u_acc.shape == (B, gamma) and u_smp.shape == (B,)
+    acc = np.empty(B, dtype=np.int32)
+    out = np.empty((B, gamma + 1), dtype=np.int32)
+    new_ctx = np.empty(B, dtype=np.int32) if ctx_len is not None else None
+    nt = nthreads or hardware_threads()
+    rc = _load().oracle_spec_accept(
+        _ptr(p, np.float32), _ptr(q, np.float32), _ptr(draft_tok, np.int32), _ptr(u_acc, np.float32),
+        _ptr(u_smp, np.float32), B, gamma, V, _ptr(ctx_len, np.int32), _ptr(acc, np.int32), _ptr(out, np.int32),
+        _ptr(new_ctx, np.int32), nt)
+    if rc != 0:
+        raise RuntimeError(f"oracle_spec_accept failed: {rc}")
+    return acc, out, new_ctx
