@@ -1,0 +1,260 @@
+/*
+ * nsd.h -- C ABI of the B200 verification round for M-for-N speculative decoding.
+ *
+ * One round = the target-side work on a batch that was rebuilt from the shared
+ * request pool (Algorithm 1 hands it over as PREPARE followed by RUN):
+ *   1. nsd_kv_prepare   make the KV state of every request present in this
+ *                       worker's pool region, then append the new tokens' KV;
+ *   2. nsd_verify_attn  ragged paged grouped-query attention, gamma+1 causal
+ *                       query rows per request (anchor + gamma proposals);
+ *   3. nsd_spec_accept  speculative acceptance / residual resampling / bonus.
+ * nsd_verify_round enqueues all three for every layer, with the preparation on
+ * a side stream that overlaps attention (Section 4: Run(B_k) || Prepare(B_k+1),
+ * here inside one batch: attention over resident requests || copy of the
+ * reassigned ones).
+ *
+ * Conventions
+ *  - Every function returns nsd_status; NSD_OK = 0.  Nothing throws.
+ *  - Pointers are DEVICE pointers unless the name starts with h_ (host).
+ *  - The caller owns every buffer, including the workspace the context lives
+ *    on; the library allocates no device memory.  nsd_create additionally owns
+ *    one CUDA side stream, a few events and a small pinned host staging area,
+ *    released by nsd_destroy.
+ *  - Device work is enqueued on the cudaStream_t passed as `stream` (cast to
+ *    void*; 0 = legacy default stream) and the call returns after enqueue.
+ *  - Host-visible arguments are validated before anything is launched; a
+ *    failing call launches nothing.  Device-side index checks (block ids read
+ *    from device tables) never fault: a bad id is replaced by block 0, the
+ *    event is recorded in a status word, and nsd_get_status reports it.
+ *  - bf16 tensors are raw 16-bit patterns.  Compiled for sm_100a only.
+ *
+ * KV pool layout (bf16):
+ *     kv_pool[slab][block][kv][kv_head][slot][dim]
+ *       slab    in [0, num_slabs)     logical layer l lives in slab l % num_slabs
+ *       block   in [0, num_blocks)    ids < region_b_begin: region A (sources),
+ *                                     the rest: region B (this worker's bank);
+ *                                     Appendix E.2's separate block ranges
+ *       kv      0 = K, 1 = V
+ *       slot    in [0, block_size)    token position inside the block
+ *   so one (slab, block) is one contiguous chunk of 2*Hkv*block_size*head_dim
+ *   bf16 (64 KiB at the Qwen3-8B shape), and one (slab, block, kv, head) tile is
+ *   one contiguous block_size*head_dim chunk (4 KiB).
+ *   num_slabs == num_layers in production; a smaller num_slabs lets a
+ *   benchmark run all logical layers over fewer physical slabs.
+ *
+ * Block tables: request r owns entries kv_indices[kv_indptr[r] .. kv_indptr[r+1]);
+ * token position t of the request lives in block kv_indices[kv_indptr[r] + t /
+ * block_size], slot t % block_size (Section 3, "KV cache organization").
+ * ctx_len[r] counts the KV entries committed BEFORE the round; the round
+ * appends gamma+1 entries at positions ctx_len[r] .. ctx_len[r]+gamma, and
+ * query row i of the request sees keys [0, ctx_len[r] + i].
+ */
+#ifndef NSD_H_
+#define NSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    NSD_OK = 0,
+    NSD_ERR_INVALID_ARG = 1,   /* null pointer, negative size, malformed host table          */
+    NSD_ERR_OUT_OF_RANGE = 2,  /* gamma, batch, layer or vocab outside the configured limits */
+    NSD_ERR_CAPACITY = 3,      /* workspace, table or partial-result capacity exceeded       */
+    NSD_ERR_UNSUPPORTED = 4,   /* head_dim / block_size / group size this build has no kernel for */
+    NSD_ERR_CUDA = 5,          /* a CUDA runtime call failed; see nsd_last_error             */
+    NSD_ERR_DEVICE_FAULT = 6,  /* a kernel met an out-of-range index in a device table       */
+    NSD_ERR_NOT_PLANNED = 7    /* nsd_verify_attn / nsd_verify_round before nsd_verify_plan  */
+} nsd_status;
+
+typedef struct nsd_ctx nsd_ctx;
+
+typedef struct {
+    int32_t num_layers;        /* logical layers of one round                            */
+    int32_t num_slabs;         /* physical layer slabs in the pool, 1..num_layers        */
+    int32_t num_q_heads;
+    int32_t num_kv_heads;      /* divides num_q_heads                                    */
+    int32_t head_dim;          /* 64 or 128                                              */
+    int32_t block_size;        /* 16                                                     */
+    int32_t num_blocks;        /* blocks per slab, both regions                          */
+    int32_t region_b_begin;    /* blocks [0,begin) = region A, [begin,num_blocks) = B    */
+    int32_t max_batch;
+    int32_t max_gamma;         /* (num_q_heads/num_kv_heads)*(max_gamma+1) <= 64         */
+    int32_t vocab_size;
+    int32_t reserved;
+    int64_t max_table_entries; /* upper bound of kv_indptr[batch]                        */
+} nsd_config;
+
+const char* nsd_status_string(nsd_status s);
+/* Text of the last failing CUDA call made through `ctx` (empty string if none). */
+const char* nsd_last_error(const nsd_ctx* ctx);
+
+/* Bytes of device workspace nsd_create needs for `cfg` (0 if cfg is invalid),
+ * and bytes of a pool with cfg->num_slabs slabs. */
+size_t nsd_workspace_bytes(const nsd_config* cfg);
+size_t nsd_kv_pool_bytes(const nsd_config* cfg);
+
+/* Builds a context on caller-provided DEVICE memory `d_workspace` (256-byte
+ * aligned, at least nsd_workspace_bytes(cfg), zero-filled by this call on the
+ * legacy default stream, which is synchronised before return).  The device
+ * current at this call owns the context. */
+nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace_bytes, nsd_ctx** out);
+nsd_status nsd_destroy(nsd_ctx* ctx);
+
+/*
+ * Host-side planning for one batch (the scheduler knows the lengths: a frozen
+ * batch carries membership and expected state versions, Appendix F.3).
+ * Validates lengths and tables, cuts every request's key range into chunks
+ * (split-KV), orders the chunks longest first and uploads the work lists on
+ * `stream`.  Must precede nsd_verify_attn / nsd_verify_round for that batch.
+ *   h_ctx_len      [batch]    committed KV entries, >= 0
+ *   h_kv_indptr    [batch+1]  non-decreasing, entry count of request r must
+ *                             cover ceil((ctx_len[r]+gamma+1)/block_size)
+ *   h_is_migrated  [batch]    nullable; 1 = reassigned to this worker this
+ *                             round (its KV arrives through the gather)
+ *   chunk_blocks   0 = choose; else the split-KV chunk length in blocks (even)
+ * Errors: INVALID_ARG (null, negative length, short table), OUT_OF_RANGE
+ * (batch > max_batch, gamma outside [1,max_gamma]), CAPACITY (table entries or
+ * split count beyond the workspace).  batch == 0 is a valid empty plan.
+ */
+nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
+                           const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
+                           void* stream);
+
+/*
+ * KV-state preparation (Section 3 "fragmented copies"; Section 5 / Appendix E.2:
+ * the destination bank is filled before Run) for layers
+ * [layer_begin, layer_begin+layer_count):
+ *   gather  for j in [0, n_mig_blocks): whole block mig_src[j] -> block
+ *           mig_dst[j] (tail slots included; sources are left untouched).  The
+ *           list is the concatenation, over the reassigned requests, of their
+ *           ceil(ctx_len/block_size) (source, destination) block pairs;
+ *   append  K/V of token t of request r written at position ctx_len[r]+t
+ *           through the block table (the append-dominant update of Section 3).
+ * Per layer the gather is enqueued before the append.
+ *   kv_pool     in/out
+ *   mig_src / mig_dst  int32 [n_mig_blocks]; n_mig_blocks == 0 skips the
+ *               gather (pointers may then be null)
+ *   k_new,v_new bf16 [num_layers][batch*(gamma+1)][num_kv_heads][head_dim],
+ *               indexed by logical layer; both null skips the append
+ *   is_migrated nullable uint8 [batch]; append_subset: 0 = every request,
+ *               1 = only requests with is_migrated == 0, 2 = only == 1
+ *               (1 and 2 need is_migrated)
+ * Destination and append blocks must be unique per request, else the result is
+ * undefined (not checked).  Errors: INVALID_ARG, OUT_OF_RANGE (layers, gamma,
+ * batch).  A bad block id on the device is skipped and reported by
+ * nsd_get_status as DEVICE_FAULT.
+ */
+nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
+                          const int32_t* mig_src, const int32_t* mig_dst, int32_t batch, int32_t gamma,
+                          const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices,
+                          const void* k_new, const void* v_new, const uint8_t* is_migrated,
+                          int32_t append_subset, int32_t layer_begin, int32_t layer_count, void* stream);
+
+/*
+ * Verification attention for one logical layer (Appendix G.2: the target
+ * processes anchor + proposal tokens; attention itself is softmax(q K^T /
+ * sqrt(head_dim)) V, q head h reading kv head h / (num_q_heads/num_kv_heads)).
+ * Uses the batch last given to nsd_verify_plan; ctx_len / kv_indptr must hold
+ * the same values on the device.
+ *   q    bf16 [batch*(gamma+1)][num_q_heads][head_dim]   (this layer's rows)
+ *   o    bf16 same shape (written for the requests of `subset`)
+ *   lse  nullable fp32 [batch*(gamma+1)][num_q_heads], natural-log sum-exp
+ *   subset  0 = all requests, 1 = resident only, 2 = reassigned only
+ * bf16 inputs, fp32 accumulation, bf16 output.
+ */
+nsd_status nsd_verify_attn(nsd_ctx* ctx, const void* kv_pool, const void* q, void* o, float* lse,
+                           int32_t batch, int32_t gamma, const int32_t* ctx_len, const int64_t* kv_indptr,
+                           const int32_t* kv_indices, int32_t layer, int32_t subset, void* stream);
+
+/*
+ * Speculative acceptance (the rule Section 1 cites: Leviathan et al. 2023,
+ * Chen et al. 2023).  For request r: accept draft i while
+ * u_acc[r][i] < min(1, p[r][i][x_i] / q[r][i][x_i]) (strict; q == 0 accepts iff
+ * p > 0), n = number accepted; if n < gamma draw y from max(0, p[r][n] - q[r][n])
+ * (from p[r][n] itself if that residual is empty), else draw the bonus token
+ * from p[r][gamma]; draws are inverse-CDF over token ids: smallest k whose
+ * cumulative weight exceeds u_smp[r] * total.  Compares and sums are done in
+ * fp64 on the fp32 inputs; the residual is an fp32 subtraction.
+ *   p  fp32 [batch][gamma+1][vocab]   q  fp32 [batch][gamma][vocab]
+ *   draft_tok int32 [batch][gamma]    u_acc fp32 [batch][gamma]   u_smp fp32 [batch]
+ *   acc_len int32 [batch]             out_tok int32 [batch][gamma+1]: accepted
+ *   drafts, then y, then -1 padding
+ *   ctx_len / new_ctx_len  nullable pair: new_ctx_len[r] = ctx_len[r] + 1 + n
+ * Errors: INVALID_ARG, OUT_OF_RANGE (gamma, batch, vocab < 1).  A draft token
+ * outside [0, vocab) counts as rejected and is reported as DEVICE_FAULT.
+ */
+nsd_status nsd_spec_accept(nsd_ctx* ctx, const float* p, const float* q, const int32_t* draft_tok,
+                           const float* u_acc, const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab,
+                           const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len,
+                           void* stream);
+
+/* Per-round tensors of nsd_verify_round; every pointer on the device. */
+typedef struct {
+    void* kv_pool;
+    int64_t n_mig_blocks;         /* (source, destination) block pairs of the gather */
+    const int32_t* mig_src;
+    const int32_t* mig_dst;
+    int32_t batch;
+    int32_t gamma;
+    const int32_t* ctx_len;
+    const int64_t* kv_indptr;
+    const int32_t* kv_indices;
+    const uint8_t* is_migrated;   /* required when n_mig_blocks > 0 */
+    const void* k_new;            /* [num_layers][rows][Hkv][D] */
+    const void* v_new;
+    const void* q;                /* [num_layers][rows][Hq][D]  */
+    void* o;                      /* [num_layers][rows][Hq][D]  */
+    const float* p;               /* acceptance inputs, as nsd_spec_accept */
+    const float* q_draft;
+    const int32_t* draft_tok;
+    const float* u_acc;
+    const float* u_smp;
+    int32_t* acc_len;
+    int32_t* out_tok;
+    int32_t* new_ctx_len;         /* nullable */
+} nsd_round_args;
+
+/*
+ * One whole verification round (every step above, every logical layer),
+ * enqueued with the preparation overlapped behind attention: per layer the
+ * side stream gathers and appends the reassigned requests while `stream`
+ * appends and attends the resident ones, then waits for the layer's copy event
+ * (the KVReady condition of Eq. (F.3)) and attends the reassigned ones;
+ * acceptance follows the last layer.  With num_slabs < num_layers the gather of
+ * layer l also waits for attention of layer l - num_slabs.  Needs a plan for
+ * this batch.  Returns after enqueue; `stream` carries the completion.
+ */
+nsd_status nsd_verify_round(nsd_ctx* ctx, const nsd_round_args* args, void* stream);
+
+/*
+ * The same round for a caller whose per-round tensors live in HOST memory
+ * (pinned for full speed): every input of `h` except kv_pool is copied to the
+ * matching buffer of `d` on `stream`, the round runs, and o, acc_len, out_tok
+ * (and new_ctx_len when both are non-null) are copied back into `h`'s buffers;
+ * the call synchronises `stream` before returning.  `h->kv_pool` is ignored:
+ * the pool is worker state that stays on the device.  h_* table arguments of
+ * the plan are taken from `h` (ctx_len, kv_indptr, is_migrated), so no separate
+ * nsd_verify_plan call is needed.  Bytes moved are written to the two counters
+ * when non-null.
+ */
+nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const nsd_round_args* d,
+                                 int64_t total_table_entries, void* stream, int64_t* h2d_bytes,
+                                 int64_t* d2h_bytes);
+
+/* Number of kernels this library has launched through `ctx` since creation. */
+int64_t nsd_launch_count(const nsd_ctx* ctx);
+
+/* Synchronises the device work of `ctx` on `stream` and the side stream, then
+ * reads the status word: NSD_OK, or NSD_ERR_DEVICE_FAULT with the first
+ * offending request index (or -1) in *first_bad_request (nullable).  The word
+ * is cleared by the call. */
+nsd_status nsd_get_status(nsd_ctx* ctx, void* stream, int32_t* first_bad_request);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NSD_H_ */

@@ -1,0 +1,537 @@
+// C ABI of the verification-round library: context, host-side validation and
+// planning, and the stream choreography of the fused round (Section 4: the
+// preparation of state overlaps model execution; Eq. (F.3): a batch runs only
+// once its KV state is ready).  See include/nsd.h for the contract.
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "nsd_internal.h"
+
+using namespace nsd;
+
+struct nsd_ctx {
+    nsd_config cfg;
+    Shape shape;
+    int device;
+    // device workspace carve-up
+    char* ws;
+    size_t ws_bytes;
+    int32_t* d_status;       // [4]
+    int32_t* d_counters;     // [max_batch * Hkv]
+    AttnItem* d_items_all;   // [max_items]
+    AttnItem* d_items_split; // [max_items]  resident items then reassigned items
+    float* d_part_ml;        // [part_slots * Hkv * Mmax * 2]
+    float* d_part_acc;       // [part_slots * Hkv * Mmax * D]
+    int64_t max_items, part_slots;
+    int32_t m_max;
+    // pinned staging for the plan
+    AttnItem* h_items;       // [2 * max_items]
+    int32_t* h_status;       // [4]
+    // current plan
+    bool planned;
+    int32_t plan_batch, plan_gamma;
+    int32_t n_all, n_res, n_mig_items;
+    // streams / events
+    cudaStream_t side;
+    cudaEvent_t ev_start, ev_side_done, ev_plan_free;
+    std::vector<cudaEvent_t> ev_prep, ev_attn;
+    int64_t launches;
+    char err[256];
+};
+
+namespace {
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+bool config_ok(const nsd_config* c) {
+    if (!c) return false;
+    if (c->num_layers < 1 || c->num_slabs < 1 || c->num_slabs > c->num_layers) return false;
+    if (c->num_q_heads < 1 || c->num_kv_heads < 1 || c->num_q_heads % c->num_kv_heads) return false;
+    if (c->num_blocks < 1 || c->region_b_begin < 0 || c->region_b_begin > c->num_blocks) return false;
+    if (c->max_batch < 1 || c->max_gamma < 1 || c->vocab_size < 1 || c->max_table_entries < 1) return false;
+    return true;
+}
+bool config_supported(const nsd_config* c) {
+    if (c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->block_size != 16) return false;
+    if (c->max_gamma > 31) return false;
+    if ((c->num_q_heads / c->num_kv_heads) * (c->max_gamma + 1) > 64) return false;
+    return true;
+}
+
+struct Layout {
+    size_t status, counters, items_all, items_split, part_ml, part_acc, total;
+    int64_t max_items, part_slots;
+    int32_t m_max;
+};
+
+Layout make_layout(const nsd_config* c) {
+    Layout L{};
+    L.m_max = (c->num_q_heads / c->num_kv_heads) * (c->max_gamma + 1);
+    // An item covers at least kMinChunkBlocks blocks unless it is a request's only or last chunk.
+    L.part_slots = std::max<int64_t>(4LL * c->max_batch, 1024);
+    L.max_items = (int64_t)c->max_batch + L.part_slots;
+    size_t off = 0;
+    L.status = off;      off = align_up(off + 4 * sizeof(int32_t), 256);
+    L.counters = off;    off = align_up(off + (size_t)c->max_batch * c->num_kv_heads * sizeof(int32_t), 256);
+    L.items_all = off;   off = align_up(off + (size_t)L.max_items * sizeof(AttnItem), 256);
+    L.items_split = off; off = align_up(off + (size_t)L.max_items * sizeof(AttnItem), 256);
+    L.part_ml = off;     off = align_up(off + (size_t)L.part_slots * c->num_kv_heads * L.m_max * 2 * sizeof(float), 256);
+    L.part_acc = off;    off = align_up(off + (size_t)L.part_slots * c->num_kv_heads * L.m_max * c->head_dim * sizeof(float), 256);
+    L.total = off;
+    return L;
+}
+
+nsd_status cuda_fail(nsd_ctx* ctx, cudaError_t e, const char* what) {
+    if (ctx) snprintf(ctx->err, sizeof ctx->err, "%s: %s", what, cudaGetErrorString(e));
+    return NSD_ERR_CUDA;
+}
+#define NSD_CUDA(ctx, call)                                         \
+    do {                                                            \
+        cudaError_t e__ = (call);                                   \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, #call);  \
+    } while (0)
+
+uint16_t* slab_ptr(const nsd_ctx* ctx, void* pool, int layer) {
+    return static_cast<uint16_t*>(pool) + (int64_t)(layer % ctx->cfg.num_slabs) * ctx->shape.slab_elems();
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* nsd_status_string(nsd_status s) {
+    switch (s) {
+        case NSD_OK: return "ok";
+        case NSD_ERR_INVALID_ARG: return "invalid argument";
+        case NSD_ERR_OUT_OF_RANGE: return "argument out of configured range";
+        case NSD_ERR_CAPACITY: return "capacity exceeded";
+        case NSD_ERR_UNSUPPORTED: return "unsupported shape";
+        case NSD_ERR_CUDA: return "CUDA runtime error";
+        case NSD_ERR_DEVICE_FAULT: return "out-of-range index met on the device";
+        case NSD_ERR_NOT_PLANNED: return "no plan for this batch";
+    }
+    return "unknown";
+}
+
+const char* nsd_last_error(const nsd_ctx* ctx) { return ctx ? ctx->err : ""; }
+
+size_t nsd_workspace_bytes(const nsd_config* cfg) {
+    if (!config_ok(cfg) || !config_supported(cfg)) return 0;
+    return make_layout(cfg).total;
+}
+
+size_t nsd_kv_pool_bytes(const nsd_config* cfg) {
+    if (!config_ok(cfg)) return 0;
+    return (size_t)cfg->num_slabs * cfg->num_blocks * 2 * cfg->num_kv_heads * cfg->block_size * cfg->head_dim * 2;
+}
+
+nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace_bytes, nsd_ctx** out) {
+    if (!out) return NSD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!config_ok(cfg) || !d_workspace) return NSD_ERR_INVALID_ARG;
+    if (!config_supported(cfg)) return NSD_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(d_workspace) % 256) return NSD_ERR_INVALID_ARG;
+    const Layout L = make_layout(cfg);
+    if (workspace_bytes < L.total) return NSD_ERR_CAPACITY;
+
+    nsd_ctx* ctx = new (std::nothrow) nsd_ctx();
+    if (!ctx) return NSD_ERR_CAPACITY;
+    ctx->cfg = *cfg;
+    ctx->shape = Shape{cfg->num_slabs, cfg->num_blocks, cfg->num_q_heads, cfg->num_kv_heads, cfg->head_dim, cfg->block_size};
+    ctx->ws = static_cast<char*>(d_workspace);
+    ctx->ws_bytes = L.total;
+    ctx->d_status = reinterpret_cast<int32_t*>(ctx->ws + L.status);
+    ctx->d_counters = reinterpret_cast<int32_t*>(ctx->ws + L.counters);
+    ctx->d_items_all = reinterpret_cast<AttnItem*>(ctx->ws + L.items_all);
+    ctx->d_items_split = reinterpret_cast<AttnItem*>(ctx->ws + L.items_split);
+    ctx->d_part_ml = reinterpret_cast<float*>(ctx->ws + L.part_ml);
+    ctx->d_part_acc = reinterpret_cast<float*>(ctx->ws + L.part_acc);
+    ctx->max_items = L.max_items;
+    ctx->part_slots = L.part_slots;
+    ctx->m_max = L.m_max;
+    ctx->planned = false;
+    ctx->launches = 0;
+    ctx->err[0] = 0;
+    ctx->h_items = nullptr;
+    ctx->h_status = nullptr;
+    ctx->side = nullptr;
+    ctx->ev_start = ctx->ev_side_done = ctx->ev_plan_free = nullptr;
+
+    auto fail = [&](cudaError_t e, const char* what) {
+        nsd_status s = cuda_fail(ctx, e, what);
+        fprintf(stderr, "nsd_create: %s\n", ctx->err);
+        nsd_destroy(ctx);
+        return s;
+    };
+    cudaError_t e;
+    if ((e = cudaGetDevice(&ctx->device)) != cudaSuccess) return fail(e, "cudaGetDevice");
+    // zero the bookkeeping part of the workspace (status, counters, work lists); partials need no init
+    if ((e = cudaMemset(ctx->ws, 0, L.part_ml)) != cudaSuccess) return fail(e, "cudaMemset(workspace)");
+    if ((e = cudaDeviceSynchronize()) != cudaSuccess) return fail(e, "cudaDeviceSynchronize");
+    if ((e = cudaMallocHost(&ctx->h_items, 2 * (size_t)L.max_items * sizeof(AttnItem))) != cudaSuccess) return fail(e, "cudaMallocHost(items)");
+    if ((e = cudaMallocHost(&ctx->h_status, 4 * sizeof(int32_t))) != cudaSuccess) return fail(e, "cudaMallocHost(status)");
+    if ((e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking)) != cudaSuccess) return fail(e, "cudaStreamCreate");
+    if ((e = cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+    if ((e = cudaEventCreateWithFlags(&ctx->ev_side_done, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+    if ((e = cudaEventCreateWithFlags(&ctx->ev_plan_free, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+    ctx->ev_prep.assign(cfg->num_layers, nullptr);
+    ctx->ev_attn.assign(cfg->num_layers, nullptr);
+    for (int l = 0; l < cfg->num_layers; ++l) {
+        if ((e = cudaEventCreateWithFlags(&ctx->ev_prep[l], cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+        if ((e = cudaEventCreateWithFlags(&ctx->ev_attn[l], cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+    }
+    if ((e = attn_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(attention)");
+    *out = ctx;
+    return NSD_OK;
+}
+
+nsd_status nsd_destroy(nsd_ctx* ctx) {
+    if (!ctx) return NSD_OK;
+    if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
+    for (auto ev : ctx->ev_prep) if (ev) cudaEventDestroy(ev);
+    for (auto ev : ctx->ev_attn) if (ev) cudaEventDestroy(ev);
+    if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
+    if (ctx->ev_side_done) cudaEventDestroy(ctx->ev_side_done);
+    if (ctx->ev_plan_free) cudaEventDestroy(ctx->ev_plan_free);
+    if (ctx->h_items) cudaFreeHost(ctx->h_items);
+    if (ctx->h_status) cudaFreeHost(ctx->h_status);
+    delete ctx;
+    return NSD_OK;
+}
+
+nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
+                           const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
+                           void* stream) {
+    if (!ctx) return NSD_ERR_INVALID_ARG;
+    if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
+    if (chunk_blocks < 0 || (chunk_blocks & 1) || chunk_blocks > 512) return NSD_ERR_INVALID_ARG;
+    if (batch > 0 && (!h_ctx_len || !h_kv_indptr)) return NSD_ERR_INVALID_ARG;
+    const int bs = ctx->cfg.block_size;
+    const int Hkv = ctx->cfg.num_kv_heads;
+    // ---- validate lengths and tables
+    std::vector<int32_t> nblk(batch);
+    int64_t total_blocks = 0;
+    for (int r = 0; r < batch; ++r) {
+        if (h_ctx_len[r] < 0 || h_kv_indptr[r] < 0 || h_kv_indptr[r + 1] < h_kv_indptr[r]) return NSD_ERR_INVALID_ARG;
+        const int64_t need = ((int64_t)h_ctx_len[r] + gamma + 1 + bs - 1) / bs;
+        if (h_kv_indptr[r + 1] - h_kv_indptr[r] < need) return NSD_ERR_INVALID_ARG;
+        if (need > INT32_MAX / 2) return NSD_ERR_OUT_OF_RANGE;
+        nblk[r] = (int32_t)need;
+        total_blocks += need;
+    }
+    if (batch > 0 && h_kv_indptr[batch] > ctx->cfg.max_table_entries) return NSD_ERR_CAPACITY;
+
+    // ---- chunk length: enough items to fill the machine several times over, long enough
+    //      that the fp32 partials of split requests stay a small fraction of the KV bytes
+    int cb = chunk_blocks;
+    if (cb == 0) {
+        const int64_t target_items = 148LL * 3 * 6;                    // SMs x resident CTAs x waves
+        int64_t want = (total_blocks * Hkv + target_items - 1) / target_items;
+        want = std::min<int64_t>(std::max<int64_t>(want, 16), 512);
+        cb = (int)((want + 1) & ~1LL);
+    }
+    auto count_slots = [&](int c) {
+        int64_t slots = 0;
+        for (int r = 0; r < batch; ++r) {
+            const int n = (nblk[r] + c - 1) / c;
+            if (n > 1) slots += n;
+        }
+        return slots;
+    };
+    while (count_slots(cb) > ctx->part_slots) {
+        if (chunk_blocks != 0 || cb >= 512) return NSD_ERR_CAPACITY;
+        cb = std::min(512, cb * 2);
+    }
+    // ---- items
+    struct Tmp { AttnItem it; int mig; };
+    std::vector<Tmp> items;
+    int32_t slot = 0;
+    for (int r = 0; r < batch; ++r) {
+        const int n = (nblk[r] + cb - 1) / cb;
+        int per = (nblk[r] + n - 1) / n;
+        per = (per + 1) & ~1;                                            // even: tiles are two blocks
+        const int n_eff = (nblk[r] + per - 1) / per;
+        const int base = n_eff > 1 ? slot : -1;
+        for (int c = 0; c < n_eff; ++c) {
+            AttnItem it{};
+            it.req = r;
+            it.blk_begin = c * per;
+            it.blk_end = std::min(nblk[r], (c + 1) * per);
+            it.part_base = base;
+            it.chunk_idx = c;
+            it.nchunks = n_eff;
+            items.push_back({it, h_is_migrated ? (h_is_migrated[r] != 0) : 0});
+        }
+        if (n_eff > 1) slot += n_eff;
+    }
+    if ((int64_t)items.size() > ctx->max_items || slot > ctx->part_slots) return NSD_ERR_CAPACITY;
+    auto longer = [](const Tmp& a, const Tmp& b) {
+        const int la = a.it.blk_end - a.it.blk_begin, lb = b.it.blk_end - b.it.blk_begin;
+        if (la != lb) return la > lb;
+        if (a.it.req != b.it.req) return a.it.req < b.it.req;
+        return a.it.chunk_idx < b.it.chunk_idx;
+    };
+    std::sort(items.begin(), items.end(), longer);
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the pinned staging may still be the source of the previous plan's copy
+    NSD_CUDA(ctx, cudaEventSynchronize(ctx->ev_plan_free));
+    const int n_all = (int)items.size();
+    int n_res = 0;
+    for (int i = 0; i < n_all; ++i) ctx->h_items[i] = items[i].it;
+    AttnItem* split = ctx->h_items + ctx->max_items;
+    for (int i = 0; i < n_all; ++i) if (!items[i].mig) split[n_res++] = items[i].it;
+    int k = n_res;
+    for (int i = 0; i < n_all; ++i) if (items[i].mig) split[k++] = items[i].it;
+    if (n_all > 0) {
+        NSD_CUDA(ctx, cudaMemcpyAsync(ctx->d_items_all, ctx->h_items, (size_t)n_all * sizeof(AttnItem), cudaMemcpyHostToDevice, st));
+        NSD_CUDA(ctx, cudaMemcpyAsync(ctx->d_items_split, split, (size_t)n_all * sizeof(AttnItem), cudaMemcpyHostToDevice, st));
+    }
+    NSD_CUDA(ctx, cudaEventRecord(ctx->ev_plan_free, st));
+    ctx->planned = true;
+    ctx->plan_batch = batch;
+    ctx->plan_gamma = gamma;
+    ctx->n_all = n_all;
+    ctx->n_res = n_res;
+    ctx->n_mig_items = n_all - n_res;
+    return NSD_OK;
+}
+
+nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
+                          const int32_t* mig_src, const int32_t* mig_dst, int32_t batch, int32_t gamma,
+                          const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices,
+                          const void* k_new, const void* v_new, const uint8_t* is_migrated,
+                          int32_t append_subset, int32_t layer_begin, int32_t layer_count, void* stream) {
+    if (!ctx || !kv_pool) return NSD_ERR_INVALID_ARG;
+    if (n_mig_blocks < 0 || layer_count < 0) return NSD_ERR_INVALID_ARG;
+    if (batch < 0 || batch > ctx->cfg.max_batch) return NSD_ERR_OUT_OF_RANGE;
+    if (layer_begin < 0 || layer_begin + (int64_t)layer_count > ctx->cfg.num_layers) return NSD_ERR_OUT_OF_RANGE;
+    const bool do_append = (k_new != nullptr) || (v_new != nullptr);
+    if (do_append) {
+        if (!k_new || !v_new || !ctx_len || !kv_indptr || !kv_indices) return NSD_ERR_INVALID_ARG;
+        if (gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
+        if (append_subset < 0 || append_subset > 2 || (append_subset != 0 && !is_migrated)) return NSD_ERR_INVALID_ARG;
+    }
+    if (n_mig_blocks > 0 && (!mig_src || !mig_dst)) return NSD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t n_pairs = n_mig_blocks;
+    const int64_t layer_rows = (int64_t)batch * (gamma + 1) * ctx->cfg.num_kv_heads * ctx->cfg.head_dim;
+    for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
+        uint16_t* slab = slab_ptr(ctx, kv_pool, l);
+        if (n_pairs > 0) {
+            NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, mig_src, mig_dst, ctx->d_status, st));
+            ctx->launches++;
+        }
+        if (do_append && batch > 0) {
+            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, ctx_len, kv_indptr, kv_indices,
+                                        static_cast<const uint16_t*>(k_new) + (int64_t)l * layer_rows,
+                                        static_cast<const uint16_t*>(v_new) + (int64_t)l * layer_rows, is_migrated,
+                                        append_subset, ctx->d_status, st));
+            ctx->launches++;
+        }
+    }
+    return NSD_OK;
+}
+
+namespace {
+nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* o, float* lse, int32_t gamma,
+                        const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices, int32_t layer,
+                        int32_t subset, cudaStream_t st) {
+    AttnLaunch a{};
+    a.shape = ctx->shape;
+    a.pool_slab = slab_ptr(ctx, const_cast<void*>(kv_pool), layer);
+    a.q = static_cast<const uint16_t*>(q);
+    a.o = static_cast<uint16_t*>(o);
+    a.lse = lse;
+    a.ctx_len = ctx_len;
+    a.kv_indptr = kv_indptr;
+    a.kv_indices = kv_indices;
+    a.gamma = gamma;
+    a.part_acc = ctx->d_part_acc;
+    a.part_ml = ctx->d_part_ml;
+    a.counters = ctx->d_counters;
+    a.status = ctx->d_status;
+    a.m_rows = (ctx->cfg.num_q_heads / ctx->cfg.num_kv_heads) * (gamma + 1);
+    if (subset == 0) { a.items = ctx->d_items_all; a.n_items = ctx->n_all; }
+    else if (subset == 1) { a.items = ctx->d_items_split; a.n_items = ctx->n_res; }
+    else { a.items = ctx->d_items_split + ctx->n_res; a.n_items = ctx->n_mig_items; }
+    if (a.n_items == 0) return NSD_OK;
+    NSD_CUDA(ctx, launch_attn(a, st));
+    ctx->launches++;
+    return NSD_OK;
+}
+}  // namespace
+
+nsd_status nsd_verify_attn(nsd_ctx* ctx, const void* kv_pool, const void* q, void* o, float* lse,
+                           int32_t batch, int32_t gamma, const int32_t* ctx_len, const int64_t* kv_indptr,
+                           const int32_t* kv_indices, int32_t layer, int32_t subset, void* stream) {
+    if (!ctx) return NSD_ERR_INVALID_ARG;
+    if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
+    if (layer < 0 || layer >= ctx->cfg.num_layers) return NSD_ERR_OUT_OF_RANGE;
+    if (subset < 0 || subset > 2) return NSD_ERR_INVALID_ARG;
+    if (!ctx->planned || ctx->plan_batch != batch || ctx->plan_gamma != gamma) return NSD_ERR_NOT_PLANNED;
+    if (batch == 0) return NSD_OK;
+    if (!kv_pool || !q || !o || !ctx_len || !kv_indptr || !kv_indices) return NSD_ERR_INVALID_ARG;
+    return attn_enqueue(ctx, kv_pool, q, o, lse, gamma, ctx_len, kv_indptr, kv_indices, layer, subset,
+                        static_cast<cudaStream_t>(stream));
+}
+
+nsd_status nsd_spec_accept(nsd_ctx* ctx, const float* p, const float* q, const int32_t* draft_tok,
+                           const float* u_acc, const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab,
+                           const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len,
+                           void* stream) {
+    if (!ctx) return NSD_ERR_INVALID_ARG;
+    if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma || vocab < 1) return NSD_ERR_OUT_OF_RANGE;
+    if (batch == 0) return NSD_OK;
+    if (!p || !q || !draft_tok || !u_acc || !u_smp || !acc_len || !out_tok) return NSD_ERR_INVALID_ARG;
+    if ((new_ctx_len != nullptr) && !ctx_len) return NSD_ERR_INVALID_ARG;
+    NSD_CUDA(ctx, launch_accept(p, q, draft_tok, u_acc, u_smp, batch, gamma, vocab, ctx_len, acc_len, out_tok,
+                                new_ctx_len, ctx->d_status, static_cast<cudaStream_t>(stream)));
+    ctx->launches++;
+    return NSD_OK;
+}
+
+nsd_status nsd_verify_round(nsd_ctx* ctx, const nsd_round_args* a, void* stream) {
+    if (!ctx || !a) return NSD_ERR_INVALID_ARG;
+    const int32_t batch = a->batch, gamma = a->gamma;
+    if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
+    if (!ctx->planned || ctx->plan_batch != batch || ctx->plan_gamma != gamma) return NSD_ERR_NOT_PLANNED;
+    if (batch == 0) return NSD_OK;
+    if (!a->kv_pool || !a->ctx_len || !a->kv_indptr || !a->kv_indices || !a->k_new || !a->v_new || !a->q || !a->o ||
+        !a->p || !a->q_draft || !a->draft_tok || !a->u_acc || !a->u_smp || !a->acc_len || !a->out_tok)
+        return NSD_ERR_INVALID_ARG;
+    if (a->n_mig_blocks < 0) return NSD_ERR_INVALID_ARG;
+    if (a->n_mig_blocks > 0 && (!a->mig_src || !a->mig_dst || !a->is_migrated)) return NSD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int L = ctx->cfg.num_layers, S = ctx->cfg.num_slabs;
+    const int Hq = ctx->cfg.num_q_heads, Hkv = ctx->cfg.num_kv_heads, D = ctx->cfg.head_dim;
+    const int64_t rows = (int64_t)batch * (gamma + 1);
+    const int64_t kv_layer = rows * Hkv * D, q_layer = rows * Hq * D;
+    const uint16_t* k_new = static_cast<const uint16_t*>(a->k_new);
+    const uint16_t* v_new = static_cast<const uint16_t*>(a->v_new);
+    const uint16_t* q = static_cast<const uint16_t*>(a->q);
+    uint16_t* o = static_cast<uint16_t*>(a->o);
+
+    const int64_t n_pairs = a->n_mig_blocks;
+    const bool overlap = n_pairs > 0;
+    if (overlap) {
+        NSD_CUDA(ctx, cudaEventRecord(ctx->ev_start, st));
+        NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_start, 0));
+    }
+    for (int l = 0; l < L; ++l) {
+        uint16_t* slab = slab_ptr(ctx, a->kv_pool, l);
+        if (overlap) {
+            // side stream: copy + append of the reassigned requests of layer l
+            if (l >= S) NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_attn[l - S], 0));
+            NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, a->mig_src, a->mig_dst, ctx->d_status, ctx->side));
+            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
+                                        k_new + l * kv_layer, v_new + l * kv_layer, a->is_migrated, 2, ctx->d_status, ctx->side));
+            NSD_CUDA(ctx, cudaEventRecord(ctx->ev_prep[l], ctx->side));
+            ctx->launches += 2;
+            // main stream: resident requests, then the reassigned ones once their state is ready
+            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
+                                        k_new + l * kv_layer, v_new + l * kv_layer, a->is_migrated, 1, ctx->d_status, st));
+            ctx->launches++;
+            nsd_status s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
+                                        a->kv_indptr, a->kv_indices, l, 1, st);
+            if (s != NSD_OK) return s;
+            NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_prep[l], 0));
+            s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
+                             a->kv_indptr, a->kv_indices, l, 2, st);
+            if (s != NSD_OK) return s;
+            if (l + S < L) NSD_CUDA(ctx, cudaEventRecord(ctx->ev_attn[l], st));
+        } else {
+            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
+                                        k_new + l * kv_layer, v_new + l * kv_layer, nullptr, 0, ctx->d_status, st));
+            ctx->launches++;
+            nsd_status s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
+                                        a->kv_indptr, a->kv_indices, l, 0, st);
+            if (s != NSD_OK) return s;
+        }
+    }
+    NSD_CUDA(ctx, launch_accept(a->p, a->q_draft, a->draft_tok, a->u_acc, a->u_smp, batch, gamma, ctx->cfg.vocab_size,
+                                a->ctx_len, a->acc_len, a->out_tok, a->new_ctx_len, ctx->d_status, st));
+    ctx->launches++;
+    return NSD_OK;
+}
+
+nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const nsd_round_args* d,
+                                 int64_t total_table_entries, void* stream, int64_t* h2d_bytes,
+                                 int64_t* d2h_bytes) {
+    if (!ctx || !h || !d) return NSD_ERR_INVALID_ARG;
+    const int32_t batch = h->batch, gamma = h->gamma;
+    if (batch != d->batch || gamma != d->gamma || h->n_mig_blocks != d->n_mig_blocks) return NSD_ERR_INVALID_ARG;
+    if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
+    if (total_table_entries < 0 || total_table_entries > ctx->cfg.max_table_entries || h->n_mig_blocks < 0) return NSD_ERR_INVALID_ARG;
+    if (batch == 0) return NSD_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int L = ctx->cfg.num_layers, Hq = ctx->cfg.num_q_heads, Hkv = ctx->cfg.num_kv_heads, D = ctx->cfg.head_dim;
+    const int64_t V = ctx->cfg.vocab_size, rows = (int64_t)batch * (gamma + 1);
+    int64_t up = 0, down = 0;
+    struct Copy { const void* src; const void* dst; int64_t bytes; };
+    const Copy ups[] = {
+        {h->ctx_len, d->ctx_len, batch * 4LL},
+        {h->kv_indptr, d->kv_indptr, (batch + 1) * 8LL},
+        {h->kv_indices, d->kv_indices, total_table_entries * 4},
+        {h->is_migrated, d->is_migrated, h->is_migrated ? batch * 1LL : 0},
+        {h->mig_src, d->mig_src, h->n_mig_blocks * 4},
+        {h->mig_dst, d->mig_dst, h->n_mig_blocks * 4},
+        {h->k_new, d->k_new, L * rows * Hkv * D * 2},
+        {h->v_new, d->v_new, L * rows * Hkv * D * 2},
+        {h->q, d->q, L * rows * Hq * D * 2},
+        {h->p, d->p, (int64_t)batch * (gamma + 1) * V * 4},
+        {h->q_draft, d->q_draft, (int64_t)batch * gamma * V * 4},
+        {h->draft_tok, d->draft_tok, (int64_t)batch * gamma * 4},
+        {h->u_acc, d->u_acc, (int64_t)batch * gamma * 4},
+        {h->u_smp, d->u_smp, batch * 4LL},
+    };
+    for (const Copy& c : ups) {
+        if (c.bytes == 0) continue;
+        if (!c.src || !c.dst) return NSD_ERR_INVALID_ARG;
+    }
+    if (!h->o || !d->o || !h->acc_len || !d->acc_len || !h->out_tok || !d->out_tok) return NSD_ERR_INVALID_ARG;
+    nsd_status s = nsd_verify_plan(ctx, batch, gamma, h->ctx_len, h->kv_indptr, h->is_migrated, 0, stream);
+    if (s != NSD_OK) return s;
+    for (const Copy& c : ups) {
+        if (c.bytes == 0) continue;
+        NSD_CUDA(ctx, cudaMemcpyAsync(const_cast<void*>(c.dst), c.src, (size_t)c.bytes, cudaMemcpyHostToDevice, st));
+        up += c.bytes;
+    }
+    s = nsd_verify_round(ctx, d, stream);
+    if (s != NSD_OK) return s;
+    const Copy downs[] = {
+        {d->o, h->o, L * rows * Hq * D * 2},
+        {d->acc_len, h->acc_len, batch * 4LL},
+        {d->out_tok, h->out_tok, rows * 4},
+        {d->new_ctx_len, h->new_ctx_len, (d->new_ctx_len && h->new_ctx_len) ? batch * 4LL : 0},
+    };
+    for (const Copy& c : downs) {
+        if (c.bytes == 0) continue;
+        NSD_CUDA(ctx, cudaMemcpyAsync(const_cast<void*>(c.dst), c.src, (size_t)c.bytes, cudaMemcpyDeviceToHost, st));
+        down += c.bytes;
+    }
+    NSD_CUDA(ctx, cudaStreamSynchronize(st));
+    if (h2d_bytes) *h2d_bytes = up;
+    if (d2h_bytes) *d2h_bytes = down;
+    return NSD_OK;
+}
+
+int64_t nsd_launch_count(const nsd_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+nsd_status nsd_get_status(nsd_ctx* ctx, void* stream, int32_t* first_bad_request) {
+    if (!ctx) return NSD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    NSD_CUDA(ctx, cudaStreamSynchronize(ctx->side));
+    NSD_CUDA(ctx, cudaMemcpyAsync(ctx->h_status, ctx->d_status, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    NSD_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, 4 * sizeof(int32_t), st));
+    NSD_CUDA(ctx, cudaStreamSynchronize(st));
+    if (first_bad_request) *first_bad_request = ctx->h_status[1] - 1;
+    return ctx->h_status[0] ? NSD_ERR_DEVICE_FAULT : NSD_OK;
+}
+
+}  // extern "C"

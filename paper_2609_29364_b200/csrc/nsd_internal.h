@@ -1,0 +1,64 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "nsd.h"
+
+namespace nsd {
+
+// One unit of attention work: a range of KV blocks of one request.  The grid
+// runs one CTA per (item, kv head).
+struct __align__(16) AttnItem {
+    int32_t req;
+    int32_t blk_begin;   // first block of the chunk (index into the request's table)
+    int32_t blk_end;     // one past the last block
+    int32_t part_base;   // first partial slot of the request, -1 when it has a single chunk
+    int32_t chunk_idx;
+    int32_t nchunks;
+    int32_t pad0, pad1;
+};
+
+// Device status word: [0] = error bits, [1] = first offending request (+1; 0 = none).
+enum : int32_t { STATUS_BAD_BLOCK = 1, STATUS_BAD_TOKEN = 2 };
+
+struct Shape {
+    int32_t num_slabs, num_blocks, Hq, Hkv, D, bs;
+    __host__ __device__ int64_t tile_elems() const { return (int64_t)bs * D; }            // one (block, kv, head)
+    __host__ __device__ int64_t block_elems() const { return 2LL * Hkv * bs * D; }        // one (slab, block)
+    __host__ __device__ int64_t slab_elems() const { return (int64_t)num_blocks * block_elems(); }
+};
+
+struct AttnLaunch {
+    Shape shape;
+    const uint16_t* pool_slab;   // base of the layer's slab
+    const uint16_t* q;
+    uint16_t* o;
+    float* lse;
+    const int32_t* ctx_len;
+    const int64_t* kv_indptr;
+    const int32_t* kv_indices;
+    const AttnItem* items;
+    int32_t n_items;
+    int32_t gamma;
+    float* part_acc;             // [slot][Hkv][M][D]
+    float* part_ml;              // [slot][Hkv][M][2]
+    int32_t* counters;           // [max_batch][Hkv], zero between launches
+    int32_t* status;
+    int32_t m_rows;              // (Hq/Hkv) * (gamma+1)
+};
+
+cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const int32_t* src, const int32_t* dst,
+                          int32_t* status, cudaStream_t stream);
+cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int32_t* ctx_len,
+                          const int64_t* kv_indptr, const int32_t* kv_indices, const uint16_t* k_new,
+                          const uint16_t* v_new, const uint8_t* is_migrated, int32_t subset, int32_t* status,
+                          cudaStream_t stream);
+cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream);
+cudaError_t attn_init();          // opt in to large dynamic shared memory, once per process
+cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
+                          const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int32_t* ctx_len,
+                          int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
+                          cudaStream_t stream);
+
+}  // namespace nsd

@@ -1,0 +1,214 @@
+// Speculative acceptance (the rule Section 1 cites from Leviathan et al. 2023 and
+// Chen et al. 2023): accept draft i while u_i < min(1, p_i(x_i)/q_i(x_i)); at the
+// first rejection draw from max(0, p - q); if nothing is rejected draw the bonus
+// token from the next target row.
+//
+// One CTA per request.  Warp 0 decides the accepted length from gamma gathers;
+// the whole CTA then sweeps ONLY the one vocabulary row pair that the draw needs
+// (not all gamma+1), keeping one partial sum per 128-token segment in shared
+// memory; the segment that holds the draw is found from the segment prefix and
+// re-read (an L2 hit) to finish inside it.  All compares and sums are fp64 on the
+// fp32 inputs, the residual is a single fp32 subtraction, so decisions agree
+// with a sequential fp64 evaluation except within rounding of a CDF boundary.
+// Compile without fast-math: IEEE division and no flush-to-zero are required.
+#include "nsd_internal.h"
+
+namespace nsd {
+namespace {
+
+constexpr int kAcceptThreads = 512;
+constexpr int kSeg = 128;                       // tokens per segment = one float4 per lane
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Weight of token k for the draw: residual (fp32 subtract, clamped) or the target row.
+__device__ __forceinline__ float weight(float pv, float qv, bool residual) {
+    if (!residual) return pv;
+    const float d = __fsub_rn(pv, qv);
+    return d > 0.0f ? d : 0.0f;
+}
+
+__global__ void __launch_bounds__(kAcceptThreads)
+spec_accept_kernel(const float* __restrict__ p, const float* __restrict__ q, const int32_t* __restrict__ draft_tok,
+                   const float* __restrict__ u_acc, const float* __restrict__ u_smp, int32_t gamma, int32_t vocab,
+                   const int32_t* __restrict__ ctx_len, int32_t* __restrict__ acc_len, int32_t* __restrict__ out_tok,
+                   int32_t* __restrict__ new_ctx_len, int32_t* __restrict__ status) {
+    extern __shared__ double seg_sum[];          // [n_seg] segment sums, then exclusive prefixes
+    __shared__ int s_n, s_found_seg, s_token;
+    __shared__ double s_total;
+
+    const int r = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_warps = kAcceptThreads / 32;
+    const int n_seg = (vocab + kSeg - 1) / kSeg;
+    const float* p_req = p + (int64_t)r * (gamma + 1) * vocab;
+    const float* q_req = q + (int64_t)r * gamma * vocab;
+
+    // ---- accepted length: first i whose test fails
+    if (warp == 0) {
+        bool reject = false;
+        if (lane < gamma) {
+            const int32_t x = draft_tok[(int64_t)r * gamma + lane];
+            if ((uint32_t)x >= (uint32_t)vocab) {
+                reject = true;
+                atomicOr(status, STATUS_BAD_TOKEN);
+                atomicCAS(status + 1, 0, r + 1);
+            } else {
+                const double P = (double)p_req[(int64_t)lane * vocab + x];
+                const double Q = (double)q_req[(int64_t)lane * vocab + x];
+                const double ratio = (Q > 0.0) ? P / Q : (P > 0.0 ? 1.0 : 0.0);
+                const double thr = ratio < 1.0 ? ratio : 1.0;
+                reject = !((double)u_acc[(int64_t)r * gamma + lane] < thr);
+            }
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, reject);
+        if (lane == 0) s_n = m ? (__ffs(m) - 1) : gamma;
+    }
+    __syncthreads();
+    const int n = s_n;
+    const float* prow = p_req + (int64_t)n * vocab;
+    const float* qrow = q_req + (int64_t)(n < gamma ? n : 0) * vocab;   // unused when n == gamma
+    bool residual = n < gamma;
+    const bool vec_ok = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(q)) % 16 == 0);
+
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        // ---- pass 1: one sum per segment
+        for (int s = warp; s < n_seg; s += n_warps) {
+            const int k0 = s * kSeg + lane * 4;
+            double acc = 0.0;
+            if (vec_ok) {
+                if (k0 < vocab) {
+                    const float4 pv = __ldg(reinterpret_cast<const float4*>(prow + k0));
+                    float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (residual) qv = __ldg(reinterpret_cast<const float4*>(qrow + k0));
+                    acc = (double)weight(pv.x, qv.x, residual);
+                    acc += (double)weight(pv.y, qv.y, residual);
+                    acc += (double)weight(pv.z, qv.z, residual);
+                    acc += (double)weight(pv.w, qv.w, residual);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (k0 + j < vocab) acc += (double)weight(prow[k0 + j], residual ? qrow[k0 + j] : 0.f, residual);
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) seg_sum[s] = acc;
+        }
+        __syncthreads();
+        // ---- exclusive prefix over segments (warp 0, lanes own consecutive runs)
+        if (warp == 0) {
+            const int per = (n_seg + 31) / 32;
+            const int b = lane * per, e = min(b + per, n_seg);
+            double local = 0.0;
+            for (int s = b; s < e; ++s) local += seg_sum[s];
+            double incl = local;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            double run = incl - local;
+            for (int s = b; s < e; ++s) {
+                const double v = seg_sum[s];
+                seg_sum[s] = run;
+                run += v;
+            }
+            const double total = __shfl_sync(0xffffffffu, incl, 31);
+            if (lane == 0) {
+                s_total = total;
+                s_found_seg = n_seg;
+            }
+        }
+        __syncthreads();
+        if (residual && s_total == 0.0) {       // empty residual: draw from the target row instead
+            residual = false;
+            __syncthreads();
+            continue;
+        }
+        break;
+    }
+
+    const double total = s_total;
+    const double t = (double)u_smp[r] * total;
+    // ---- first segment whose inclusive prefix exceeds t
+    for (int s = tid; s < n_seg; s += kAcceptThreads) {
+        const double incl = (s + 1 < n_seg) ? seg_sum[s + 1] : total;
+        if (incl > t) {
+            atomicMin(&s_found_seg, s);
+            break;                               // a thread's later segments are larger
+        }
+    }
+    __syncthreads();
+
+    // ---- finish inside the segment (warp 0); walk on if rounding left nothing there
+    if (warp == 0) {
+        int token = -1;
+        for (int s = s_found_seg; s < n_seg && token < 0; ++s) {
+            const int k0 = s * kSeg + lane * 4;
+            float w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                w[j] = (k0 + j < vocab) ? weight(prow[k0 + j], residual ? qrow[k0 + j] : 0.f, residual) : 0.f;
+            const double mine = (double)w[0] + (double)w[1] + (double)w[2] + (double)w[3];
+            double incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            double c = seg_sum[s] + (incl - mine);
+            int hit = -1;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                c += (double)w[j];
+                if (hit < 0 && k0 + j < vocab && c > t) hit = k0 + j;
+            }
+            const unsigned m = __ballot_sync(0xffffffffu, hit >= 0);
+            if (m) token = __shfl_sync(0xffffffffu, hit, __ffs(m) - 1);
+        }
+        if (token < 0 && lane == 0) {            // t not exceeded anywhere: last token with positive weight
+            for (int k = vocab - 1; k >= 0; --k)
+                if (weight(prow[k], residual ? qrow[k] : 0.f, residual) > 0.f) {
+                    token = k;
+                    break;
+                }
+        }
+        if (lane == 0) s_token = token;
+    }
+    __syncthreads();
+
+    if (tid <= gamma) {
+        int32_t v = -1;
+        if (tid < n) v = draft_tok[(int64_t)r * gamma + tid];
+        else if (tid == n) v = s_token;
+        out_tok[(int64_t)r * (gamma + 1) + tid] = v;
+    }
+    if (tid == 0) {
+        acc_len[r] = n;
+        if (new_ctx_len && ctx_len) new_ctx_len[r] = ctx_len[r] + 1 + n;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
+                          const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int32_t* ctx_len,
+                          int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
+                          cudaStream_t stream) {
+    if (batch <= 0) return cudaSuccess;
+    const int n_seg = (vocab + kSeg - 1) / kSeg;
+    const size_t smem = (size_t)(n_seg + 1) * sizeof(double);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(spec_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    spec_accept_kernel<<<batch, kAcceptThreads, smem, stream>>>(p, q, draft_tok, u_acc, u_smp, gamma, vocab, ctx_len,
+                                                              acc_len, out_tok, new_ctx_len, status);
+    return cudaGetLastError();
+}
+
+}  // namespace nsd

@@ -1,0 +1,408 @@
+// Verification attention: gamma+1 causal query rows per request over a paged,
+// ragged KV cache with grouped-query heads (Appendix G.2: the target processes
+// the anchor token plus the proposal tokens in one pass; Section 3: the KV state
+// spans non-contiguous blocks addressed through a block map).
+//
+// Shape of the work.  For one request and one kv head, the (gamma+1) rows of the
+// G = Hq/Hkv query heads that share the kv head are stacked into one M x D tile
+// (M = G*(gamma+1) = 20 at gamma 4), so every K/V byte is read from HBM once and
+// feeds all M rows through the tensor cores.  The arithmetic intensity is only
+// ~20-36 flop per KV byte, so the kernel is bound by HBM bandwidth; the tensor
+// cores (mma.sync m16n8k16, bf16 in / fp32 accumulate) keep the math off the
+// critical path.
+//
+// Parallelisation (split-KV).  The host plan cuts each request's block range into
+// chunks and orders (chunk) items longest first; the grid is one CTA per
+// (item, kv head), scheduled by the hardware in that order.  A CTA has one warp
+// per 16-row m-tile.  K/V tiles of 32 keys stream global -> shared through a
+// cp.async ring (16-byte pieces, XOR-swizzled so ldmatrix is conflict free).
+// Each warp keeps an online softmax (running max / sum in registers, quad
+// shuffles) over its rows.  A request with one chunk writes bf16 output directly;
+// otherwise the CTA stores its unnormalised fp32 partial (max, sum, acc) and the
+// LAST CTA to finish that (request, head) -- decided by an atomic counter, no
+// waiting -- merges all partials in chunk order and writes the output.
+//
+// Masking.  Row i sees keys [0, ctx + i].  Only tiles that reach past ctx need
+// the mask.  Slots past ctx+gamma in the last block may hold anything (NaN
+// included): scores there are replaced by -inf with a select, and the V rows of
+// those slots are zeroed in shared memory, so 0 * NaN never reaches an
+// accumulator.
+#include <cuda_bf16.h>
+
+#include "nsd_internal.h"
+
+namespace nsd {
+namespace {
+
+constexpr int kBlockSize = 16;      // keys per pool block
+constexpr int kTileKeys = 32;       // keys per pipeline stage (two pool blocks)
+constexpr int kStages = 4;
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Byte offset of 16-byte piece `chunk` of row `row` in a swizzled [rows][D] bf16 tile.
+template <int D>
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+    return (uint32_t)(row * (D * 2) + ((chunk ^ (row & 7)) << 4));
+}
+
+template <int D, int NMT>
+struct Smem {
+    static constexpr int kTileBytes = kTileKeys * D * 2;            // K (or V) of one stage
+    static constexpr int kQBytes = NMT * 16 * D * 2;
+    static constexpr int kMaxChunkBlocks = 512;
+    static constexpr int kBytes = kQBytes + kStages * 2 * kTileBytes + kMaxChunkBlocks * 4;
+};
+
+template <int D, int NMT>
+__global__ void __launch_bounds__(NMT * 32)
+verify_attn_kernel(const AttnLaunch a) {
+    constexpr int NT = NMT * 32;                  // threads
+    constexpr int CPR = D / 8;                    // 16-byte pieces per row
+    constexpr int KSTEPS = D / 16;                // k-steps of Q K^T
+    constexpr int DT = D / 8;                     // n-tiles of P V
+    using SM = Smem<D, NMT>;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* q_s = smem;
+    unsigned char* kv_s = smem + SM::kQBytes;
+    int32_t* blk_s = reinterpret_cast<int32_t*>(smem + SM::kQBytes + kStages * 2 * SM::kTileBytes);
+    __shared__ int s_last;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int Hkv = a.shape.Hkv, Hq = a.shape.Hq, G = Hq / Hkv;
+    const int item_idx = blockIdx.x / Hkv;
+    const int head = blockIdx.x - item_idx * Hkv;
+    const AttnItem it = a.items[item_idx];
+    const int r = it.req;
+    const int gamma = a.gamma;
+    const int ctx = a.ctx_len[r];
+    const int n_total = ctx + gamma + 1;          // keys that exist after the append
+    const int M = a.m_rows;
+    const int64_t table0 = a.kv_indptr[r];
+    const int n_blk = it.blk_end - it.blk_begin;
+    const int n_tiles = (n_blk + 1) >> 1;
+
+    // ---- block ids of the chunk -> shared (bad ids are replaced by block 0 and reported)
+    for (int i = tid; i < n_blk; i += NT) {
+        int32_t b = a.kv_indices[table0 + it.blk_begin + i];
+        if ((uint32_t)b >= (uint32_t)a.shape.num_blocks) {
+            atomicOr(a.status, STATUS_BAD_BLOCK);
+            atomicCAS(a.status + 1, 0, r + 1);
+            b = 0;
+        }
+        blk_s[i] = b;
+    }
+    // ---- Q rows -> shared (row m = i*G + j is query row i of head head*G + j); padding rows are zero
+    for (int c = tid; c < NMT * 16 * CPR; c += NT) {
+        const int m = c / CPR, ch = c - m * CPR;
+        const uint32_t dst = smem_u32(q_s) + swz<D>(m, ch);
+        if (m < M) {
+            const int i = m / G, j = m - i * G;
+            const uint16_t* src = a.q + (((int64_t)r * (gamma + 1) + i) * Hq + head * G + j) * D + ch * 8;
+            cp_async16(dst, src);
+        } else {
+            *reinterpret_cast<int4*>(q_s + swz<D>(m, ch)) = make_int4(0, 0, 0, 0);
+        }
+    }
+    __syncthreads();                              // blk_s visible before tiles are issued
+
+    const int64_t tile_elems = (int64_t)kBlockSize * D;
+    const uint16_t* k_base = a.pool_slab + (int64_t)head * tile_elems;
+    const uint16_t* v_base = k_base + (int64_t)Hkv * tile_elems;
+    const int64_t block_elems = a.shape.block_elems();
+
+    auto issue_tile = [&](int t) {
+        if (t < n_tiles) {
+            unsigned char* ks = kv_s + (t % kStages) * 2 * SM::kTileBytes;
+            unsigned char* vs = ks + SM::kTileBytes;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int bi = 2 * t + half;
+                if (bi < n_blk) {
+                    const int64_t off = (int64_t)blk_s[bi] * block_elems;
+                    for (int c = tid; c < kBlockSize * CPR; c += NT) {
+                        const int row = c / CPR, ch = c - row * CPR;
+                        const uint32_t so = swz<D>(half * kBlockSize + row, ch);
+                        cp_async16(smem_u32(ks) + so, k_base + off + c * 8);
+                        cp_async16(smem_u32(vs) + so, v_base + off + c * 8);
+                    }
+                } else {                           // no such block: V must be finite (zero); K is masked
+                    for (int c = tid; c < kBlockSize * CPR; c += NT) {
+                        const int row = c / CPR, ch = c - row * CPR;
+                        *reinterpret_cast<int4*>(vs + swz<D>(half * kBlockSize + row, ch)) = make_int4(0, 0, 0, 0);
+                    }
+                }
+            }
+        }
+        cp_async_commit();
+    };
+
+#pragma unroll
+    for (int s = 0; s < kStages - 1; ++s) issue_tile(s);
+
+    // ---- per-warp state: rows g and g+8 of m-tile `warp`
+    const int g = lane >> 2, tq = lane & 3;
+    const int m_lo = warp * 16 + g, m_hi = m_lo + 8;
+    const int lim_lo = ctx + min(m_lo / G, gamma);      // last visible key of the row
+    const int lim_hi = ctx + min(m_hi / G, gamma);
+    const float sc = rsqrtf((float)D) * kLog2e;          // scores in the log2 domain
+    float o_acc[DT][4];
+#pragma unroll
+    for (int i = 0; i < DT; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
+    float mx_lo = -INFINITY, mx_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+    uint32_t qf[KSTEPS][4];
+
+    const int key0_chunk = it.blk_begin * kBlockSize;
+    for (int t = 0; t < n_tiles; ++t) {
+        cp_async_wait<kStages - 2>();
+        __syncthreads();
+        issue_tile(t + kStages - 1);
+        if (t == 0) {                                  // Q landed with the first group
+#pragma unroll
+            for (int kk = 0; kk < KSTEPS; ++kk) {
+                const int mi = lane >> 3;
+                ldmatrix_x4(qf[kk], smem_u32(q_s) + swz<D>(warp * 16 + (mi & 1) * 8 + (lane & 7), kk * 2 + (mi >> 1)));
+            }
+        }
+        unsigned char* ks = kv_s + (t % kStages) * 2 * SM::kTileBytes;
+        unsigned char* vs = ks + SM::kTileBytes;
+        const int key0 = key0_chunk + t * kTileKeys;
+        const bool need_mask = key0 + kTileKeys > ctx + 1;   // some key of the tile is hidden from some row
+        if (key0 + kTileKeys > n_total) {                    // slots that hold no token: zero their V rows
+            for (int c = tid; c < kTileKeys * CPR; c += NT) {
+                const int row = c / CPR, ch = c - row * CPR;
+                if (key0 + row >= n_total) *reinterpret_cast<int4*>(vs + swz<D>(row, ch)) = make_int4(0, 0, 0, 0);
+            }
+            __syncthreads();
+        }
+
+        // ---- S = Q K^T (16 rows x 32 keys per warp)
+        float s[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < KSTEPS; ++kk) {
+            const int mi = lane >> 3;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t kf[4];
+                ldmatrix_x4(kf, smem_u32(ks) + swz<D>(half * 16 + (mi >> 1) * 8 + (lane & 7), kk * 2 + (mi & 1)));
+                mma_bf16(s[half * 2 + 0], qf[kk], kf[0], kf[1]);
+                mma_bf16(s[half * 2 + 1], qf[kk], kf[2], kf[3]);
+            }
+        }
+        // ---- scale, mask, online softmax
+        float tmax_lo = -INFINITY, tmax_hi = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int key = key0 + nt * 8 + tq * 2 + e;
+                float vlo = s[nt][e] * sc, vhi = s[nt][2 + e] * sc;
+                if (need_mask) {
+                    vlo = key <= lim_lo ? vlo : -INFINITY;
+                    vhi = key <= lim_hi ? vhi : -INFINITY;
+                }
+                s[nt][e] = vlo;
+                s[nt][2 + e] = vhi;
+                tmax_lo = fmaxf(tmax_lo, vlo);
+                tmax_hi = fmaxf(tmax_hi, vhi);
+            }
+        }
+        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(0xffffffffu, tmax_lo, 1));
+        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(0xffffffffu, tmax_lo, 2));
+        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(0xffffffffu, tmax_hi, 1));
+        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(0xffffffffu, tmax_hi, 2));
+        const float new_lo = fmaxf(mx_lo, tmax_lo), new_hi = fmaxf(mx_hi, tmax_hi);
+        const float use_lo = new_lo == -INFINITY ? 0.f : new_lo;     // nothing visible yet: avoid inf - inf
+        const float use_hi = new_hi == -INFINITY ? 0.f : new_hi;
+        const float resc_lo = exp2f(mx_lo - use_lo), resc_hi = exp2f(mx_hi - use_hi);
+        mx_lo = new_lo;
+        mx_hi = new_hi;
+        float sum_lo = 0.f, sum_hi = 0.f;
+        uint32_t pf[2][4];                               // P as A-fragments: [k-step of 16 keys]
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            const float p0 = exp2f(s[nt][0] - use_lo), p1 = exp2f(s[nt][1] - use_lo);
+            const float p2 = exp2f(s[nt][2] - use_hi), p3 = exp2f(s[nt][3] - use_hi);
+            sum_lo += p0 + p1;
+            sum_hi += p2 + p3;
+            pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
+            pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+        }
+        l_lo = l_lo * resc_lo + sum_lo;
+        l_hi = l_hi * resc_hi + sum_hi;
+#pragma unroll
+        for (int i = 0; i < DT; ++i) {
+            o_acc[i][0] *= resc_lo;
+            o_acc[i][1] *= resc_lo;
+            o_acc[i][2] *= resc_hi;
+            o_acc[i][3] *= resc_hi;
+        }
+        // ---- O += P V
+#pragma unroll
+        for (int ks16 = 0; ks16 < 2; ++ks16) {
+            const int mi = lane >> 3;
+#pragma unroll
+            for (int dp = 0; dp < DT / 2; ++dp) {
+                uint32_t vf[4];
+                ldmatrix_x4_trans(vf, smem_u32(vs) + swz<D>(ks16 * 16 + (mi & 1) * 8 + (lane & 7), dp * 2 + (mi >> 1)));
+                mma_bf16(o_acc[dp * 2 + 0], pf[ks16], vf[0], vf[1]);
+                mma_bf16(o_acc[dp * 2 + 1], pf[ks16], vf[2], vf[3]);
+            }
+        }
+    }
+    cp_async_wait<0>();
+
+    // ---- row sums across the quad
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+
+    const int64_t row_base = (int64_t)r * (gamma + 1);
+    if (it.part_base < 0) {
+        // ---- single chunk: normalise and write bf16
+#pragma unroll
+        for (int hl = 0; hl < 2; ++hl) {
+            const int m = hl ? m_hi : m_lo;
+            if (m >= M) continue;
+            const float l = hl ? l_hi : l_lo;
+            const float inv = 1.f / l;
+            const int i = m / G, j = m - i * G;
+            const int64_t orow = ((row_base + i) * Hq + head * G + j);
+            uint16_t* op = a.o + orow * D;
+#pragma unroll
+            for (int dt = 0; dt < DT; ++dt)
+                *reinterpret_cast<uint32_t*>(op + dt * 8 + tq * 2) =
+                    pack_bf16(o_acc[dt][hl * 2 + 0] * inv, o_acc[dt][hl * 2 + 1] * inv);
+            if (a.lse && tq == 0) a.lse[orow] = ((hl ? mx_hi : mx_lo) + log2f(l)) * 0.6931471805599453f;
+        }
+        return;
+    }
+
+    // ---- several chunks: store the partial, the last CTA of this (request, head) merges
+    {
+        const int64_t slot = ((int64_t)it.part_base + it.chunk_idx) * Hkv + head;
+        float* pa = a.part_acc + slot * M * D;
+        float* pm = a.part_ml + slot * M * 2;
+#pragma unroll
+        for (int hl = 0; hl < 2; ++hl) {
+            const int m = hl ? m_hi : m_lo;
+            if (m >= M) continue;
+#pragma unroll
+            for (int dt = 0; dt < DT; ++dt)
+                *reinterpret_cast<float2*>(pa + (int64_t)m * D + dt * 8 + tq * 2) =
+                    make_float2(o_acc[dt][hl * 2 + 0], o_acc[dt][hl * 2 + 1]);
+            if (tq == 0) *reinterpret_cast<float2*>(pm + m * 2) = make_float2(hl ? mx_hi : mx_lo, hl ? l_hi : l_lo);
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        int32_t* cnt = a.counters + (int64_t)r * Hkv + head;
+        const int old = atomicAdd(cnt, 1);
+        const int last = (old == it.nchunks - 1);
+        if (last) *cnt = 0;                               // ready for the next launch
+        s_last = last;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int e = tid; e < M * (D / 4); e += NT) {
+        const int m = e / (D / 4), d4 = e - m * (D / 4);
+        float mstar = -INFINITY;
+        for (int c = 0; c < it.nchunks; ++c) {
+            const int64_t slot = ((int64_t)it.part_base + c) * Hkv + head;
+            mstar = fmaxf(mstar, __ldcg(a.part_ml + (slot * M + m) * 2));
+        }
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float l = 0.f;
+        for (int c = 0; c < it.nchunks; ++c) {
+            const int64_t slot = ((int64_t)it.part_base + c) * Hkv + head;
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (slot * M + m) * 2));
+            const float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mstar);
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_acc + (slot * M + m) * D) + d4);
+            acc.x += w * v.x;
+            acc.y += w * v.y;
+            acc.z += w * v.z;
+            acc.w += w * v.w;
+            l += w * ml.y;
+        }
+        const float inv = 1.f / l;
+        const int i = m / G, j = m - i * G;
+        const int64_t orow = ((row_base + i) * Hq + head * G + j);
+        uint2 packed;
+        packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+        packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(a.o + orow * D + d4 * 4) = packed;
+        if (a.lse && d4 == 0) a.lse[orow] = (mstar + log2f(l)) * 0.6931471805599453f;
+    }
+}
+
+template <int D, int NMT>
+cudaError_t launch_one(const AttnLaunch& a, cudaStream_t stream) {
+    const int64_t grid = (int64_t)a.n_items * a.shape.Hkv;
+    verify_attn_kernel<D, NMT><<<(unsigned)grid, NMT * 32, Smem<D, NMT>::kBytes, stream>>>(a);
+    return cudaGetLastError();
+}
+
+template <int D, int NMT>
+cudaError_t init_one() {
+    return cudaFuncSetAttribute(verify_attn_kernel<D, NMT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                Smem<D, NMT>::kBytes);
+}
+
+}  // namespace
+
+cudaError_t attn_init() {
+    cudaError_t e;
+#define NSD_INIT(DD, NN) \
+    if ((e = init_one<DD, NN>()) != cudaSuccess) return e;
+    NSD_INIT(64, 1) NSD_INIT(64, 2) NSD_INIT(64, 3) NSD_INIT(64, 4)
+    NSD_INIT(128, 1) NSD_INIT(128, 2) NSD_INIT(128, 3) NSD_INIT(128, 4)
+#undef NSD_INIT
+    return cudaSuccess;
+}
+
+cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
+    if (a.n_items <= 0) return cudaSuccess;
+    const int nmt = (a.m_rows + 15) / 16;
+#define NSD_CASE(DD, NN) \
+    if (a.shape.D == DD && nmt == NN) return launch_one<DD, NN>(a, stream);
+    NSD_CASE(64, 1) NSD_CASE(64, 2) NSD_CASE(64, 3) NSD_CASE(64, 4)
+    NSD_CASE(128, 1) NSD_CASE(128, 2) NSD_CASE(128, 3) NSD_CASE(128, 4)
+#undef NSD_CASE
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace nsd

@@ -1,0 +1,121 @@
+"""GPU parity: the fused nsd_verify_round (side-stream prepare overlapped with
+attention, every layer, then acceptance) and its host-buffer variant against the
+oracle sequence gather -> append -> attention per layer, then acceptance."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workload as W
+from nsd_testlib import (DeviceBatch, accept_compare, attn_mismatch, dev, guarded_pool, guards_intact, host_u16,
+                         make_context, stack_layers)
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_round(cfg, meta, pool0, k_new, v_new, q, acc_in):
+    pool = pool0.copy()
+    outs = []
+    for l in range(cfg.num_layers):
+        oracle.kv_prepare(pool, meta.mig_indptr, meta.mig_src, meta.mig_dst, meta.ctx_len, meta.kv_indptr,
+                          meta.kv_indices, k_new, v_new, cfg.gamma, layer_begin=l, layer_count=1)
+        outs.append(oracle.verify_attn(pool, q[l], meta.ctx_len, meta.kv_indptr, meta.kv_indices, cfg.gamma, layer=l))
+    acc, out, new_ctx = oracle.spec_accept(*acc_in, meta.ctx_len)
+    return pool, outs, acc, out, new_ctx
+
+
+def _run_round(cfg, slabs, host_variant=False, repeat=1):
+    meta = W.make_batch_meta(cfg)
+    pool0 = np.stack([W.pool_layer(cfg, meta, s) for s in range(slabs)])
+    k_new, v_new = stack_layers(cfg, meta, "kv")
+    q = stack_layers(cfg, meta, "q")
+    acc_in = W.accept_inputs(cfg)
+    p, qd, tok, ua, us = acc_in
+    ctx = make_context(cfg, meta, num_slabs=slabs)
+    db = DeviceBatch(meta)
+    buf, pool = guarded_pool(pool0)
+    B, g1 = cfg.batch, cfg.gamma + 1
+    d = dict(kv_pool=pool, n_mig_blocks=db.n_mig_blocks, mig_src=db.mig_src, mig_dst=db.mig_dst, batch=B,
+             gamma=cfg.gamma, ctx_len=db.ctx_len, kv_indptr=db.kv_indptr, kv_indices=db.kv_indices,
+             is_migrated=db.is_migrated, k_new=dev(k_new), v_new=dev(v_new), q=dev(q),
+             o=torch.full(q.shape, 0x7FC0, dtype=torch.int16, device="cuda:0"), p=dev(p), q_draft=dev(qd),
+             draft_tok=dev(tok), u_acc=dev(ua), u_smp=dev(us),
+             acc_len=torch.full((B,), -7, dtype=torch.int32, device="cuda:0"),
+             out_tok=torch.full((B, g1), -7, dtype=torch.int32, device="cuda:0"),
+             new_ctx_len=torch.full((B,), -7, dtype=torch.int32, device="cuda:0"))
+    stream = torch.cuda.Stream()
+    if host_variant:
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a.view(np.int16) if a.dtype == np.uint16 else a)).pin_memory()
+        h = dict(kv_pool=None, n_mig_blocks=db.n_mig_blocks, mig_src=pin(meta.mig_src) if db.n_mig_blocks else None,
+                 mig_dst=pin(meta.mig_dst) if db.n_mig_blocks else None, batch=B, gamma=cfg.gamma,
+                 ctx_len=pin(meta.ctx_len), kv_indptr=pin(meta.kv_indptr), kv_indices=pin(meta.kv_indices),
+                 is_migrated=pin(meta.is_migrated), k_new=pin(k_new), v_new=pin(v_new), q=pin(q),
+                 o=torch.zeros(q.shape, dtype=torch.int16).pin_memory(), p=pin(p), q_draft=pin(qd), draft_tok=pin(tok),
+                 u_acc=pin(ua), u_smp=pin(us), acc_len=torch.zeros(B, dtype=torch.int32).pin_memory(),
+                 out_tok=torch.zeros((B, g1), dtype=torch.int32).pin_memory(),
+                 new_ctx_len=torch.zeros(B, dtype=torch.int32).pin_memory())
+        # the device copies start as garbage: everything must arrive through the call
+        for k in ("ctx_len", "kv_indptr", "kv_indices", "is_migrated", "k_new", "v_new", "q", "p", "q_draft",
+                  "draft_tok", "u_acc", "u_smp"):
+            d[k] = torch.zeros_like(d[k])
+        if db.n_mig_blocks:
+            d["mig_src"], d["mig_dst"] = torch.zeros_like(d["mig_src"]), torch.zeros_like(d["mig_dst"])
+        with torch.cuda.stream(stream):
+            for _ in range(repeat):
+                up, down = ctx.nsd_verify_round_host(ctx.round_args(**h), ctx.round_args(**d), int(meta.kv_indptr[-1]),
+                                                     stream=stream)
+        assert up > p.nbytes and down >= q.nbytes
+        o_gpu, acc_g, out_g, new_g = h["o"].numpy().view(np.uint16), h["acc_len"].numpy(), h["out_tok"].numpy(), h["new_ctx_len"].numpy()
+    else:
+        with torch.cuda.stream(stream):
+            ctx.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, meta.is_migrated, cfg.gamma, stream=stream)
+            for _ in range(repeat):
+                ctx.nsd_verify_round(ctx.round_args(**d), stream=stream)
+        stream.synchronize()
+        o_gpu, acc_g, out_g, new_g = host_u16(d["o"]), d["acc_len"].cpu().numpy(), d["out_tok"].cpu().numpy(), d["new_ctx_len"].cpu().numpy()
+    rc, bad = ctx.nsd_get_status(stream=stream)
+    assert rc == 0, (rc, bad)
+    assert guards_intact(buf)
+    want_pool, outs, acc_r, out_r, new_r = _oracle_round(cfg, meta, pool0, k_new, v_new, q, acc_in)
+    assert np.array_equal(host_u16(pool).reshape(want_pool.shape), want_pool)
+    for l in range(cfg.num_layers):
+        bad, max_abs, max_rel = attn_mismatch(o_gpu[l], outs[l])
+        assert bad == 0, (l, bad, max_abs, max_rel)
+    rep = accept_compare(p, qd, tok, ua, us, acc_g, out_g, acc_r, out_r)
+    assert rep["len_exact"] == cfg.batch
+    assert (new_g == new_r).all()
+    return ctx
+
+
+MULTI = W.RoundConfig("round_multi", batch=10, gamma=4, num_layers=5, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                      block_size=16, vocab=3000, ctx_dist=("uniform", 1, 1200), frac_reassigned=0.4, seed=81)
+NOMIG = W.RoundConfig("round_nomig", batch=6, gamma=6, num_layers=2, num_q_heads=8, num_kv_heads=2, head_dim=64,
+                      block_size=16, vocab=500, ctx_dist=("uniform", 1, 300), frac_reassigned=0.0, seed=82)
+ALLMIG = W.RoundConfig("round_allmig", batch=6, gamma=8, num_layers=3, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                       block_size=16, vocab=500, ctx_dist=("uniform", 1, 500), frac_reassigned=1.0, seed=83)
+
+
+def test_tiny_config_round():
+    _run_round(W.CONFIGS["tiny"], 1)
+
+
+@pytest.mark.parametrize("cfg,slabs", [(MULTI, 5), (MULTI, 2), (NOMIG, 2), (ALLMIG, 1), (ALLMIG, 3)],
+                         ids=["multi", "multi_alias2", "nomig", "allmig_alias1", "allmig"])
+def test_multi_layer_round(cfg, slabs):
+    _run_round(cfg, slabs)
+
+
+def test_round_twice_gives_the_same_state():
+    """The round is idempotent on its inputs (what the benchmark relies on)."""
+    _run_round(MULTI, 2, repeat=3)
+
+
+def test_host_buffer_round():
+    _run_round(MULTI, 2, host_variant=True)
+    _run_round(W.CONFIGS["tiny"], 1, host_variant=True, repeat=2)
+
+
+def test_launch_count_matches_the_choreography():
+    ctx = _run_round(MULTI, 5)
+    # per layer: gather + reassigned append + resident append + 2 attention launches; one acceptance
+    assert ctx.nsd_launch_count() == 5 * 5 + 1
