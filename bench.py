@@ -1,0 +1,457 @@
+#!/usr/bin/env python
+"""Benchmark of the B200 verification round (the benchmark spec metric: verify-round
+req/s and tokens/s at the Qwen3-8B shape, HBM GB/s against the B200 peak).
+
+One step = one whole verification round through the C ABI on one batch of
+synthetic input: for each of the 36 logical layers the KV-state preparation
+(block gather of the reassigned requests + append of the gamma+1 new tokens),
+the ragged paged GQA attention, and finally the speculative acceptance.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload knee_b512]
+    python bench.py --impl reference ...      # the CPU oracle, on host cores
+
+Prints ONE JSON line (rank 0).  N > 1 (under torchrun) runs one independent
+batch per GPU -- the path has no exchange step -- and reports the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workload as W  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="knee_b512", choices=list(W.CONFIGS))
+    ap.add_argument("--slabs", type=int, default=0, help="physical layer slabs (0 = as many as fit in 80%% of free memory)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target CPU time of the oracle sample")
+    ap.add_argument("--batch", type=int, default=0, help="profiling only: override the batch size (not a bench line)")
+    ap.add_argument("--layers", type=int, default=0, help="profiling only: override the layer count (not a bench line)")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------- algorithmic bytes
+def algorithmic_bytes(cfg: W.RoundConfig, meta: W.BatchMeta, acc_len=None):
+    """Bytes the method itself must move (per layer unless noted): every KV byte of
+    every visible key once, Q read and O written once, each gathered block read
+    and written once, each appended row read and written once, and for the
+    acceptance the one vocabulary row (pair) the draw needs."""
+    kv_tok = 2 * cfg.num_kv_heads * cfg.head_dim * 2
+    block_bytes = kv_tok * cfg.block_size
+    keys = int((meta.ctx_len.astype(np.int64) + cfg.gamma + 1).sum())
+    attn = keys * kv_tok + cfg.rows * cfg.num_q_heads * cfg.head_dim * 2 * 2
+    gather = int(len(meta.mig_src)) * block_bytes * 2
+    append = cfg.rows * kv_tok * 2
+    if acc_len is None:
+        accept = cfg.batch * cfg.vocab * 4 * 2
+    else:
+        accept = int(((acc_len < cfg.gamma) + 1).sum()) * cfg.vocab * 4
+    accept += 12 * cfg.batch * cfg.gamma
+    per_round = cfg.num_layers * (attn + gather + append) + accept
+    return dict(attn_per_layer=attn, gather_per_layer=gather, append_per_layer=append, accept=accept, round=per_round)
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.gpu_id = gpu_id
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="nsd_clocks_", suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), power_w_max=float(max(pw)),
+                       reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------- oracle arm
+def oracle_sample(cfg, meta, host, target_seconds):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload and
+    extrapolates to one whole round.  Returns (seconds per round, description, cores)."""
+    import oracle
+
+    cores = oracle.hardware_threads()
+    L, B = cfg.num_layers, cfg.batch
+    pool = host["pool_slab"][None].copy()
+    t0 = time.perf_counter()
+    oracle.kv_prepare(pool, meta.mig_indptr, meta.mig_src, meta.mig_dst, meta.ctx_len, meta.kv_indptr, meta.kv_indices,
+                      host["k_new"][:1], host["v_new"][:1], cfg.gamma, layer_begin=0, layer_count=1)
+    t_prep = time.perf_counter() - t0
+    order = np.random.default_rng(cfg.seed).permutation(B).astype(np.int32)
+    n_probe = min(B, cores)
+    t0 = time.perf_counter()
+    oracle.verify_attn(pool, host["q"][0], meta.ctx_len, meta.kv_indptr, meta.kv_indices, cfg.gamma, layer=0,
+                       req_list=np.ascontiguousarray(order[:n_probe]))
+    t_probe = time.perf_counter() - t0
+    # spend about target_seconds: first more requests of layer 0, then further layers' query rows
+    want = n_probe * max(target_seconds, t_probe) / max(t_probe, 1e-3)           # request-layers affordable
+    n_attn = int(min(B, max(n_probe, want)))
+    n_layers = int(min(L, max(1, want // max(n_attn, 1))))
+    sel = np.ascontiguousarray(order[:n_attn])
+    keys_all = float((meta.ctx_len.astype(np.int64) + cfg.gamma + 1).sum())
+    keys_sel = float((meta.ctx_len[sel].astype(np.int64) + cfg.gamma + 1).sum())
+    t0 = time.perf_counter()
+    for l in range(n_layers):
+        oracle.verify_attn(pool, host["q"][l], meta.ctx_len, meta.kv_indptr, meta.kv_indices, cfg.gamma, layer=0, req_list=sel)
+    t_attn = time.perf_counter() - t0
+    t_attn_layer = t_attn / n_layers * keys_all / keys_sel   # attention cost is proportional to visible keys
+    t0 = time.perf_counter()
+    oracle.spec_accept(host["p"], host["q_draft"], host["draft_tok"], host["u_acc"], host["u_smp"], meta.ctx_len)
+    t_acc = time.perf_counter() - t0
+    t_round = L * (t_prep + t_attn_layer) + t_acc
+    desc = (f"kv-prepare: 1 of {L} layers, all {B} requests ({t_prep:.2f}s); attention: {n_layers} layer(s) x {len(sel)} of {B} "
+            f"requests ({t_attn:.2f}s, scaled by visible keys); acceptance: all {B} requests ({t_acc:.2f}s); "
+            f"round time extrapolated x{L} layers")
+    return t_round, desc, cores
+
+
+def host_inputs(cfg, meta, layers_needed=None, with_pool=True):
+    L = cfg.num_layers
+    host = {}
+    if with_pool:
+        host["pool_slab"] = W.pool_layer(cfg, meta, 0, poison=False)
+    kv = [W.new_kv(cfg, meta, l) for l in range(L)]
+    host["k_new"] = np.stack([a for a, _ in kv])
+    host["v_new"] = np.stack([b for _, b in kv])
+    host["q"] = np.stack([W.queries(cfg, meta, l) for l in range(L)])
+    host["p"], host["q_draft"], host["draft_tok"], host["u_acc"], host["u_smp"] = W.accept_inputs(cfg)
+    return host
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle on the host cores, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = pick_config(args)
+    meta = W.make_batch_meta(cfg)
+    host = host_inputs(cfg, meta)
+    per_step = max(2.0, min(args.cpu_seconds, 150.0 / max(1, args.steps + args.warmup)))
+    times, desc, cores = [], "", 1
+    for i in range(args.warmup + args.steps):
+        t, desc, cores = oracle_sample(cfg, meta, host, per_step)
+        if i >= args.warmup:
+            times.append(t)
+    t_round = float(np.mean(times))
+    value = cfg.batch / t_round
+    line = {
+        "impl": "reference", "metric": "verify_round_requests_per_s", "value": value, "unit": "req/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_round * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg, meta, None),
+        "cpu_baseline": {"value": value, "unit": "req/s", "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "req/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def pick_config(args) -> W.RoundConfig:
+    cfg = W.CONFIGS[args.workload]
+    if args.batch or args.layers:
+        cfg = W.RoundConfig(**{**cfg.__dict__, "batch": args.batch or cfg.batch, "num_layers": args.layers or cfg.num_layers,
+                               "name": cfg.name + "_REDUCED_FOR_PROFILING"})
+    return cfg
+
+
+def workload_config(cfg, meta, slabs):
+    base = cfg.name.replace("_REDUCED_FOR_PROFILING", "")
+    return {
+        "workload": f"{cfg.name} (BASELINE.json configs[{list(W.CONFIGS).index(base)}])", "batch": cfg.batch,
+        "gamma": cfg.gamma, "layers": cfg.num_layers, "physical_layer_slabs": slabs,
+        "heads": f"{cfg.num_q_heads}q/{cfg.num_kv_heads}kv x {cfg.head_dim}", "block_size": cfg.block_size,
+        "vocab": cfg.vocab, "ctx": list(cfg.ctx_dist), "mean_ctx": float(meta.ctx_len.mean()),
+        "reassigned_requests": int(meta.n_mig), "pool_blocks_per_layer": int(meta.num_blocks),
+        "l2_policy": "inputs larger than L2: each layer slab is several GB, consecutive layers use different slabs",
+    }
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_29364_b200 as nsd
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    n_gpus = world
+
+    base = pick_config(args)
+    cfg = base if rank == 0 else W.RoundConfig(**{**base.__dict__, "seed": base.seed + 1000 * rank})
+    meta = W.make_batch_meta(cfg)
+    host = host_inputs(cfg, meta)
+    L, B, g1 = cfg.num_layers, cfg.batch, cfg.gamma + 1
+    slab_bytes = meta.num_blocks * cfg.block_elems * 2
+    free, _total = torch.cuda.mem_get_info(device)
+    other = host["p"].nbytes + host["q_draft"].nbytes + 3 * host["q"].nbytes
+    slabs = args.slabs or int(min(L, max(1, (0.8 * free - other) // slab_bytes)))
+    if L > 1 and slabs < 2:
+        raise SystemExit("not enough device memory for two layer slabs")
+
+    def dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a.view(np.int16) if a.dtype == np.uint16 else a)).to(device)
+
+    ctx = nsd.VerifyContext(num_layers=L, num_slabs=slabs, num_q_heads=cfg.num_q_heads, num_kv_heads=cfg.num_kv_heads,
+                            head_dim=cfg.head_dim, block_size=cfg.block_size, num_blocks=meta.num_blocks,
+                            region_b_begin=meta.region_b_begin, max_batch=B, max_gamma=cfg.gamma, vocab_size=cfg.vocab,
+                            max_table_entries=int(meta.kv_indptr[-1]), device=str(device))
+    pool = torch.empty((slabs, meta.num_blocks * cfg.block_elems), dtype=torch.int16, device=device)
+    pool[0].copy_(torch.from_numpy(host["pool_slab"].reshape(-1).view(np.int16)))
+    for s in range(1, slabs):
+        pool[s].copy_(pool[0])          # every slab starts from the same bytes; the appends make the layers differ
+    d = dict(kv_pool=pool, n_mig_blocks=len(meta.mig_src), mig_src=dev(meta.mig_src), mig_dst=dev(meta.mig_dst),
+             batch=B, gamma=cfg.gamma, ctx_len=dev(meta.ctx_len), kv_indptr=dev(meta.kv_indptr),
+             kv_indices=dev(meta.kv_indices), is_migrated=dev(meta.is_migrated), k_new=dev(host["k_new"]),
+             v_new=dev(host["v_new"]), q=dev(host["q"]), o=torch.zeros(host["q"].shape, dtype=torch.int16, device=device),
+             p=dev(host["p"]), q_draft=dev(host["q_draft"]), draft_tok=dev(host["draft_tok"]), u_acc=dev(host["u_acc"]),
+             u_smp=dev(host["u_smp"]), acc_len=torch.zeros(B, dtype=torch.int32, device=device),
+             out_tok=torch.zeros((B, g1), dtype=torch.int32, device=device),
+             new_ctx_len=torch.zeros(B, dtype=torch.int32, device=device))
+    d_args = ctx.round_args(**d)
+    stream = torch.cuda.Stream(device)
+
+    def barrier():
+        torch.cuda.synchronize(device)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def timed(fn, steps, warmup):
+        """ms per step of fn(), CUDA events on the launching stream, max over ranks."""
+        with torch.cuda.stream(stream):
+            for _ in range(warmup):
+                fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(steps):
+                fn()
+            e1.record(stream)
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1)) / steps
+
+    # ---- headline: whole rounds, inputs resident in HBM
+    with torch.cuda.stream(stream):
+        ctx.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, meta.is_migrated, cfg.gamma, stream=stream)
+    props = torch.cuda.get_device_properties(device)
+    sampler = ClockSampler("GPU-" + str(props.uuid) if getattr(props, "uuid", None) else str(local))
+    launches0 = None
+
+    def one_round():
+        ctx.nsd_verify_round(d_args, stream=stream)
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            one_round()
+    barrier()
+    launches0 = ctx.nsd_launch_count()
+    sampler.start()
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(args.steps):
+            one_round()
+        e1.record(stream)
+    barrier()
+    ms_round = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    gpu_launches = ctx.nsd_launch_count() - launches0
+    clocks = sampler.stop()
+    rc, bad = ctx.nsd_get_status(stream=stream)
+    if rc != 0:
+        raise SystemExit(f"device status {rc} (request {bad})")
+    acc_len = d["acc_len"].cpu().numpy()
+    committed = int((acc_len + 1).sum())
+    bytes_ = algorithmic_bytes(cfg, meta, acc_len)
+
+    # ---- dominant kernel alone: attention, one launch per layer, events around the launches
+    with torch.cuda.stream(stream):
+        ctx.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, None, cfg.gamma, stream=stream)
+
+    def attn_all_layers():
+        for l in range(L):
+            ctx.nsd_verify_attn(pool, d["q"][l], d["o"][l], None, B, cfg.gamma, d["ctx_len"], d["kv_indptr"],
+                                d["kv_indices"], layer=l, subset=0, stream=stream)
+
+    ms_attn_launch = timed(attn_all_layers, args.steps, args.warmup) / L
+    peak, peak_kind = measured_peak()
+    attn_gbs = bytes_["attn_per_layer"] / (ms_attn_launch * 1e-3) / 1e9
+
+    # ---- the other kernels alone and the round without any reassigned request (exposed prepare time)
+    def prepare_all_layers():
+        ctx.nsd_kv_prepare(pool, d["n_mig_blocks"], d["mig_src"], d["mig_dst"], B, cfg.gamma, d["ctx_len"], d["kv_indptr"],
+                           d["kv_indices"], d["k_new"], d["v_new"], stream=stream)
+
+    def accept_only():
+        ctx.nsd_spec_accept(d["p"], d["q_draft"], d["draft_tok"], d["u_acc"], d["u_smp"], B, cfg.gamma, cfg.vocab,
+                            d["ctx_len"], d["acc_len"], d["out_tok"], d["new_ctx_len"], stream=stream)
+
+    ms_prepare_layer = timed(prepare_all_layers, max(2, args.steps // 2), 1) / L
+    ms_accept = timed(accept_only, max(5, args.steps), 2)
+    nomig = ctx.round_args(**{**d, "n_mig_blocks": 0, "mig_src": None, "mig_dst": None, "is_migrated": None})
+    ms_round_nomig = timed(lambda: ctx.nsd_verify_round(nomig, stream=stream), max(2, args.steps // 2), 1)
+    exposed_ms = ms_round - ms_round_nomig
+    gather_bar_ms = L * bytes_["gather_per_layer"] / (0.7 * NOMINAL_HBM_GBS * 1e9) * 1e3
+
+    # ---- end to end: per-round tensors start in pinned host memory, results read back
+    e2e = None
+    if not args.no_e2e:
+        def pin(a):
+            return torch.from_numpy(np.ascontiguousarray(a.view(np.int16) if a.dtype == np.uint16 else a)).pin_memory()
+
+        h = dict(kv_pool=None, n_mig_blocks=len(meta.mig_src), mig_src=pin(meta.mig_src), mig_dst=pin(meta.mig_dst),
+                 batch=B, gamma=cfg.gamma, ctx_len=pin(meta.ctx_len), kv_indptr=pin(meta.kv_indptr),
+                 kv_indices=pin(meta.kv_indices), is_migrated=pin(meta.is_migrated), k_new=pin(host["k_new"]),
+                 v_new=pin(host["v_new"]), q=pin(host["q"]), o=torch.zeros(host["q"].shape, dtype=torch.int16).pin_memory(),
+                 p=pin(host["p"]), q_draft=pin(host["q_draft"]), draft_tok=pin(host["draft_tok"]),
+                 u_acc=pin(host["u_acc"]), u_smp=pin(host["u_smp"]), acc_len=torch.zeros(B, dtype=torch.int32).pin_memory(),
+                 out_tok=torch.zeros((B, g1), dtype=torch.int32).pin_memory(),
+                 new_ctx_len=torch.zeros(B, dtype=torch.int32).pin_memory())
+        h_args = ctx.round_args(**h)
+        moved = {}
+
+        def host_round():
+            moved["up"], moved["down"] = ctx.nsd_verify_round_host(h_args, d_args, int(meta.kv_indptr[-1]), stream=stream)
+
+        e2e_steps = max(2, min(args.steps, 5))
+        host_round()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            host_round()                       # synchronises the stream before returning
+        barrier()
+        ms_e2e = max_over_ranks((time.perf_counter() - t0) * 1e3) / e2e_steps
+        assert np.array_equal(h["acc_len"].numpy(), acc_len), "host-buffer round disagrees with the device-buffer round"
+        e2e = {"value": n_gpus * B / (ms_e2e * 1e-3), "unit": "req/s", "ms_per_step": ms_e2e, "steps": e2e_steps,
+               "h2d_bytes_per_step": int(moved["up"]), "d2h_bytes_per_step": int(moved["down"]),
+               "api": "nsd_verify_round_host (pinned host buffers; the KV pool is worker state and stays in HBM)"}
+
+    # ---- the oracle on the host cores (rank 0, N = 1 only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        t_round_cpu, desc, cores = oracle_sample(cfg, meta, host, args.cpu_seconds)
+        cpu_baseline = {"value": B / t_round_cpu, "unit": "req/s", "cores": cores, "kind": "oracle", "sample": desc,
+                        "seconds_per_round_extrapolated": t_round_cpu}
+
+    if rank == 0:
+        round_gbs = bytes_["round"] / (ms_round * 1e-3) / 1e9
+        line = {
+            "metric": "verify_round_requests_per_s", "value": n_gpus * B / (ms_round * 1e-3), "unit": "req/s",
+            "n_gpus": n_gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_round,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(cfg, meta, slabs),
+            "committed_tokens_per_s": n_gpus * committed / (ms_round * 1e-3),
+            "verified_rows_per_s": n_gpus * cfg.rows / (ms_round * 1e-3),
+            "mean_accepted_len": float(acc_len.mean()),
+            "roofline": {"kernel": "verify_attn_kernel (one launch per layer, timed alone)", "bound": "hbm",
+                         "achieved": attn_gbs, "peak": peak, "peak_kind": f"{peak_kind} copy bandwidth",
+                         "unit": "GB/s", "frac": attn_gbs / peak, "frac_of_nominal_8TBs": attn_gbs / NOMINAL_HBM_GBS,
+                         "traffic": None, "bytes_per_launch": bytes_["attn_per_layer"], "ms_per_launch": ms_attn_launch},
+            "round_roofline": {"bound": "hbm", "achieved": round_gbs, "peak": peak, "unit": "GB/s",
+                               "frac": round_gbs / peak, "frac_of_nominal_8TBs": round_gbs / NOMINAL_HBM_GBS,
+                               "algorithmic_bytes_per_round": bytes_["round"]},
+            "breakdown_ms": {"attn_per_layer_alone": ms_attn_launch, "prepare_per_layer_alone": ms_prepare_layer,
+                             "accept_alone": ms_accept, "round_without_reassignment": ms_round_nomig,
+                             "exposed_prepare": exposed_ms, "exposed_prepare_bar": gather_bar_ms,
+                             "prepare_GBs_alone": (bytes_["gather_per_layer"] + bytes_["append_per_layer"]) / (ms_prepare_layer * 1e-3) / 1e9,
+                             "accept_GBs_alone": bytes_["accept"] / (ms_accept * 1e-3) / 1e9},
+            "e2e": e2e, "gpu_launches": int(gpu_launches), "clocks": clocks, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

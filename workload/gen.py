@@ -227,12 +227,15 @@ def pool_layer(cfg: RoundConfig, meta: BatchMeta, layer: int, poison: bool = Tru
     pool = np.full((meta.num_blocks, 2, Hkv, bs, D), fill, dtype=np.uint16)
     n_home = int(meta.home_indptr[-1])
     if n_home:
-        data = _normal_bf16(_rng(cfg.seed, "pool", layer), (n_home, 2, Hkv, bs, D))
+        rng = _rng(cfg.seed, "pool", layer)
+        step = 1024                                   # home blocks per draw (part of the recipe: fixes the stream)
+        for b0 in range(0, n_home, step):
+            b1 = min(n_home, b0 + step)
+            pool[meta.home_blocks[b0:b1]] = _normal_bf16(rng, (b1 - b0, 2, Hkv, bs, D))
         tail = meta.ctx_len.astype(np.int64) % bs
         for r in np.nonzero(tail)[0]:
-            last = int(meta.home_indptr[r + 1]) - 1
-            data[last, :, :, int(tail[r]):, :] = fill
-        pool[meta.home_blocks] = data
+            last = int(meta.home_blocks[int(meta.home_indptr[r + 1]) - 1])
+            pool[last, :, :, int(tail[r]):, :] = fill
     return pool
 
 
