@@ -46,6 +46,7 @@ struct AttnLaunch {
     int32_t* counters;           // [max_batch][Hkv], zero between launches
     int32_t* status;
     int32_t m_rows;              // (Hq/Hkv) * (gamma+1)
+    int32_t tune_stages;         // experiment knob: 0 = default pipeline depth
 };
 
 cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const int32_t* src, const int32_t* dst,

@@ -36,7 +36,6 @@ namespace {
 
 constexpr int kBlockSize = 16;      // keys per pool block
 constexpr int kTileKeys = 32;       // keys per pipeline stage (two pool blocks)
-constexpr int kStages = 4;
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -75,26 +74,30 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
     return (uint32_t)(row * (D * 2) + ((chunk ^ (row & 7)) << 4));
 }
 
-template <int D, int NMT>
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int D, int kStages>
 struct Smem {
     static constexpr int kTileBytes = kTileKeys * D * 2;            // K (or V) of one stage
-    static constexpr int kQBytes = NMT * 16 * D * 2;
     static constexpr int kMaxChunkBlocks = 512;
-    static constexpr int kBytes = kQBytes + kStages * 2 * kTileBytes + kMaxChunkBlocks * 4;
+    static constexpr int kBytes = kStages * 2 * kTileBytes + kMaxChunkBlocks * 4;
 };
 
-template <int D, int NMT>
+template <int D, int NMT, int kStages>
 __global__ void __launch_bounds__(NMT * 32)
 verify_attn_kernel(const AttnLaunch a) {
     constexpr int NT = NMT * 32;                  // threads
     constexpr int CPR = D / 8;                    // 16-byte pieces per row
     constexpr int KSTEPS = D / 16;                // k-steps of Q K^T
     constexpr int DT = D / 8;                     // n-tiles of P V
-    using SM = Smem<D, NMT>;
+    using SM = Smem<D, kStages>;
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* q_s = smem;
-    unsigned char* kv_s = smem + SM::kQBytes;
-    int32_t* blk_s = reinterpret_cast<int32_t*>(smem + SM::kQBytes + kStages * 2 * SM::kTileBytes);
+    unsigned char* kv_s = smem;
+    int32_t* blk_s = reinterpret_cast<int32_t*>(smem + kStages * 2 * SM::kTileBytes);
     __shared__ int s_last;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -120,18 +123,6 @@ verify_attn_kernel(const AttnLaunch a) {
             b = 0;
         }
         blk_s[i] = b;
-    }
-    // ---- Q rows -> shared (row m = i*G + j is query row i of head head*G + j); padding rows are zero
-    for (int c = tid; c < NMT * 16 * CPR; c += NT) {
-        const int m = c / CPR, ch = c - m * CPR;
-        const uint32_t dst = smem_u32(q_s) + swz<D>(m, ch);
-        if (m < M) {
-            const int i = m / G, j = m - i * G;
-            const uint16_t* src = a.q + (((int64_t)r * (gamma + 1) + i) * Hq + head * G + j) * D + ch * 8;
-            cp_async16(dst, src);
-        } else {
-            *reinterpret_cast<int4*>(q_s + swz<D>(m, ch)) = make_int4(0, 0, 0, 0);
-        }
     }
     __syncthreads();                              // blk_s visible before tiles are issued
 
@@ -174,25 +165,33 @@ verify_attn_kernel(const AttnLaunch a) {
     const int m_lo = warp * 16 + g, m_hi = m_lo + 8;
     const int lim_lo = ctx + min(m_lo / G, gamma);      // last visible key of the row
     const int lim_hi = ctx + min(m_hi / G, gamma);
-    const float sc = rsqrtf((float)D) * kLog2e;          // scores in the log2 domain
+    const float sc = rsqrtf((float)D) * kLog2e;          // raw score -> log2 domain
     float o_acc[DT][4];
 #pragma unroll
     for (int i = 0; i < DT; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
     float mx_lo = -INFINITY, mx_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+    // ---- Q fragments straight from global memory (row m = i*G + j is query row i of head head*G + j;
+    //      rows past M are zero): a0/a2 = row g, a1/a3 = row g+8, columns kk*16 + {0,8} + 2*tq
     uint32_t qf[KSTEPS][4];
+    {
+        const uint16_t* q_lo = nullptr;
+        const uint16_t* q_hi = nullptr;
+        if (m_lo < M) q_lo = a.q + (((int64_t)r * (gamma + 1) + m_lo / G) * Hq + head * G + m_lo % G) * D + tq * 2;
+        if (m_hi < M) q_hi = a.q + (((int64_t)r * (gamma + 1) + m_hi / G) * Hq + head * G + m_hi % G) * D + tq * 2;
+#pragma unroll
+        for (int kk = 0; kk < KSTEPS; ++kk) {
+            qf[kk][0] = q_lo ? __ldg(reinterpret_cast<const uint32_t*>(q_lo + kk * 16)) : 0u;
+            qf[kk][1] = q_hi ? __ldg(reinterpret_cast<const uint32_t*>(q_hi + kk * 16)) : 0u;
+            qf[kk][2] = q_lo ? __ldg(reinterpret_cast<const uint32_t*>(q_lo + kk * 16 + 8)) : 0u;
+            qf[kk][3] = q_hi ? __ldg(reinterpret_cast<const uint32_t*>(q_hi + kk * 16 + 8)) : 0u;
+        }
+    }
 
     const int key0_chunk = it.blk_begin * kBlockSize;
     for (int t = 0; t < n_tiles; ++t) {
         cp_async_wait<kStages - 2>();
         __syncthreads();
         issue_tile(t + kStages - 1);
-        if (t == 0) {                                  // Q landed with the first group
-#pragma unroll
-            for (int kk = 0; kk < KSTEPS; ++kk) {
-                const int mi = lane >> 3;
-                ldmatrix_x4(qf[kk], smem_u32(q_s) + swz<D>(warp * 16 + (mi & 1) * 8 + (lane & 7), kk * 2 + (mi >> 1)));
-            }
-        }
         unsigned char* ks = kv_s + (t % kStages) * 2 * SM::kTileBytes;
         unsigned char* vs = ks + SM::kTileBytes;
         const int key0 = key0_chunk + t * kTileKeys;
@@ -220,22 +219,19 @@ verify_attn_kernel(const AttnLaunch a) {
                 mma_bf16(s[half * 2 + 1], qf[kk], kf[2], kf[3]);
             }
         }
-        // ---- scale, mask, online softmax
+        // ---- mask, online softmax (max over raw scores; the scale is folded into the exponent)
         float tmax_lo = -INFINITY, tmax_hi = -INFINITY;
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-                const int key = key0 + nt * 8 + tq * 2 + e;
-                float vlo = s[nt][e] * sc, vhi = s[nt][2 + e] * sc;
                 if (need_mask) {
-                    vlo = key <= lim_lo ? vlo : -INFINITY;
-                    vhi = key <= lim_hi ? vhi : -INFINITY;
+                    const int key = key0 + nt * 8 + tq * 2 + e;
+                    s[nt][e] = key <= lim_lo ? s[nt][e] : -INFINITY;
+                    s[nt][2 + e] = key <= lim_hi ? s[nt][2 + e] : -INFINITY;
                 }
-                s[nt][e] = vlo;
-                s[nt][2 + e] = vhi;
-                tmax_lo = fmaxf(tmax_lo, vlo);
-                tmax_hi = fmaxf(tmax_hi, vhi);
+                tmax_lo = fmaxf(tmax_lo, s[nt][e]);
+                tmax_hi = fmaxf(tmax_hi, s[nt][2 + e]);
             }
         }
         tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(0xffffffffu, tmax_lo, 1));
@@ -243,30 +239,32 @@ verify_attn_kernel(const AttnLaunch a) {
         tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(0xffffffffu, tmax_hi, 1));
         tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(0xffffffffu, tmax_hi, 2));
         const float new_lo = fmaxf(mx_lo, tmax_lo), new_hi = fmaxf(mx_hi, tmax_hi);
-        const float use_lo = new_lo == -INFINITY ? 0.f : new_lo;     // nothing visible yet: avoid inf - inf
-        const float use_hi = new_hi == -INFINITY ? 0.f : new_hi;
-        const float resc_lo = exp2f(mx_lo - use_lo), resc_hi = exp2f(mx_hi - use_hi);
+        const bool grew = (new_lo != mx_lo) || (new_hi != mx_hi);
+        const float off_lo = new_lo == -INFINITY ? 0.f : -new_lo * sc;   // nothing visible yet: avoid inf - inf
+        const float off_hi = new_hi == -INFINITY ? 0.f : -new_hi * sc;
+        if (__any_sync(0xffffffffu, grew)) {                // rescale only when some row's maximum moved
+            const float resc_lo = ex2_approx(fmaf(mx_lo, sc, off_lo)), resc_hi = ex2_approx(fmaf(mx_hi, sc, off_hi));
+            l_lo *= resc_lo;
+            l_hi *= resc_hi;
+#pragma unroll
+            for (int i = 0; i < DT; ++i) {
+                o_acc[i][0] *= resc_lo;
+                o_acc[i][1] *= resc_lo;
+                o_acc[i][2] *= resc_hi;
+                o_acc[i][3] *= resc_hi;
+            }
+        }
         mx_lo = new_lo;
         mx_hi = new_hi;
-        float sum_lo = 0.f, sum_hi = 0.f;
         uint32_t pf[2][4];                               // P as A-fragments: [k-step of 16 keys]
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
-            const float p0 = exp2f(s[nt][0] - use_lo), p1 = exp2f(s[nt][1] - use_lo);
-            const float p2 = exp2f(s[nt][2] - use_hi), p3 = exp2f(s[nt][3] - use_hi);
-            sum_lo += p0 + p1;
-            sum_hi += p2 + p3;
+            const float p0 = ex2_approx(fmaf(s[nt][0], sc, off_lo)), p1 = ex2_approx(fmaf(s[nt][1], sc, off_lo));
+            const float p2 = ex2_approx(fmaf(s[nt][2], sc, off_hi)), p3 = ex2_approx(fmaf(s[nt][3], sc, off_hi));
+            l_lo += p0 + p1;
+            l_hi += p2 + p3;
             pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
             pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
-        }
-        l_lo = l_lo * resc_lo + sum_lo;
-        l_hi = l_hi * resc_hi + sum_hi;
-#pragma unroll
-        for (int i = 0; i < DT; ++i) {
-            o_acc[i][0] *= resc_lo;
-            o_acc[i][1] *= resc_lo;
-            o_acc[i][2] *= resc_hi;
-            o_acc[i][3] *= resc_hi;
         }
         // ---- O += P V
 #pragma unroll
@@ -305,7 +303,7 @@ verify_attn_kernel(const AttnLaunch a) {
             for (int dt = 0; dt < DT; ++dt)
                 *reinterpret_cast<uint32_t*>(op + dt * 8 + tq * 2) =
                     pack_bf16(o_acc[dt][hl * 2 + 0] * inv, o_acc[dt][hl * 2 + 1] * inv);
-            if (a.lse && tq == 0) a.lse[orow] = ((hl ? mx_hi : mx_lo) + log2f(l)) * 0.6931471805599453f;
+            if (a.lse && tq == 0) a.lse[orow] = ((hl ? mx_hi : mx_lo) * sc + log2f(l)) * 0.6931471805599453f;
         }
         return;
     }
@@ -323,7 +321,7 @@ verify_attn_kernel(const AttnLaunch a) {
             for (int dt = 0; dt < DT; ++dt)
                 *reinterpret_cast<float2*>(pa + (int64_t)m * D + dt * 8 + tq * 2) =
                     make_float2(o_acc[dt][hl * 2 + 0], o_acc[dt][hl * 2 + 1]);
-            if (tq == 0) *reinterpret_cast<float2*>(pm + m * 2) = make_float2(hl ? mx_hi : mx_lo, hl ? l_hi : l_lo);
+            if (tq == 0) *reinterpret_cast<float2*>(pm + m * 2) = make_float2((hl ? mx_hi : mx_lo) * sc, hl ? l_hi : l_lo);
         }
     }
     __threadfence();
@@ -369,27 +367,30 @@ verify_attn_kernel(const AttnLaunch a) {
     }
 }
 
-template <int D, int NMT>
+template <int D, int NMT, int kStages>
 cudaError_t launch_one(const AttnLaunch& a, cudaStream_t stream) {
     const int64_t grid = (int64_t)a.n_items * a.shape.Hkv;
-    verify_attn_kernel<D, NMT><<<(unsigned)grid, NMT * 32, Smem<D, NMT>::kBytes, stream>>>(a);
+    verify_attn_kernel<D, NMT, kStages><<<(unsigned)grid, NMT * 32, Smem<D, kStages>::kBytes, stream>>>(a);
     return cudaGetLastError();
 }
 
-template <int D, int NMT>
+template <int D, int NMT, int kStages>
 cudaError_t init_one() {
-    return cudaFuncSetAttribute(verify_attn_kernel<D, NMT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                Smem<D, NMT>::kBytes);
+    return cudaFuncSetAttribute(verify_attn_kernel<D, NMT, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                Smem<D, kStages>::kBytes);
 }
+
+constexpr int kStagesD64 = 4, kStagesD128 = 3;
 
 }  // namespace
 
 cudaError_t attn_init() {
     cudaError_t e;
-#define NSD_INIT(DD, NN) \
-    if ((e = init_one<DD, NN>()) != cudaSuccess) return e;
-    NSD_INIT(64, 1) NSD_INIT(64, 2) NSD_INIT(64, 3) NSD_INIT(64, 4)
-    NSD_INIT(128, 1) NSD_INIT(128, 2) NSD_INIT(128, 3) NSD_INIT(128, 4)
+#define NSD_INIT(DD, NN, SS) \
+    if ((e = init_one<DD, NN, SS>()) != cudaSuccess) return e;
+    NSD_INIT(64, 1, kStagesD64) NSD_INIT(64, 2, kStagesD64) NSD_INIT(64, 3, kStagesD64) NSD_INIT(64, 4, kStagesD64)
+    NSD_INIT(128, 1, kStagesD128) NSD_INIT(128, 2, kStagesD128) NSD_INIT(128, 3, kStagesD128) NSD_INIT(128, 4, kStagesD128)
+    NSD_INIT(128, 2, 2) NSD_INIT(128, 2, 4)
 #undef NSD_INIT
     return cudaSuccess;
 }
@@ -397,10 +398,12 @@ cudaError_t attn_init() {
 cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
     if (a.n_items <= 0) return cudaSuccess;
     const int nmt = (a.m_rows + 15) / 16;
-#define NSD_CASE(DD, NN) \
-    if (a.shape.D == DD && nmt == NN) return launch_one<DD, NN>(a, stream);
-    NSD_CASE(64, 1) NSD_CASE(64, 2) NSD_CASE(64, 3) NSD_CASE(64, 4)
-    NSD_CASE(128, 1) NSD_CASE(128, 2) NSD_CASE(128, 3) NSD_CASE(128, 4)
+    if (a.shape.D == 128 && nmt == 2 && a.tune_stages == 2) return launch_one<128, 2, 2>(a, stream);
+    if (a.shape.D == 128 && nmt == 2 && a.tune_stages == 4) return launch_one<128, 2, 4>(a, stream);
+#define NSD_CASE(DD, NN, SS) \
+    if (a.shape.D == DD && nmt == NN) return launch_one<DD, NN, SS>(a, stream);
+    NSD_CASE(64, 1, kStagesD64) NSD_CASE(64, 2, kStagesD64) NSD_CASE(64, 3, kStagesD64) NSD_CASE(64, 4, kStagesD64)
+    NSD_CASE(128, 1, kStagesD128) NSD_CASE(128, 2, kStagesD128) NSD_CASE(128, 3, kStagesD128) NSD_CASE(128, 4, kStagesD128)
 #undef NSD_CASE
     return cudaErrorInvalidValue;
 }
