@@ -245,6 +245,49 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
                                  int64_t total_table_entries, void* stream, int64_t* h2d_bytes,
                                  int64_t* d2h_bytes);
 
+/*
+ * Attention for callers that are not allowed to allocate device memory.
+ * (No counterpart in the paper: this entry point exists for the hosts of the
+ * library, not for the method.)
+ *
+ * Who needs it: code that runs inside somebody else's memory budget (a plugin in
+ * a serving runtime that owns the allocator), a worker whose device memory was
+ * split up once at start-up and must not grow, or a latency path where an
+ * allocator call may stall behind a device-wide synchronisation.  Such a caller
+ * cannot provide the workspace nsd_create wants, so this variant of
+ * nsd_verify_attn keeps its split-KV scratch (work list, arrival counters, fp32
+ * partial results, status word) in a fixed array inside the library: about 8.1
+ * MiB of device memory that every GPU loading the library holds until the
+ * process exits.  The call itself performs no cudaMalloc / cudaFree and uses no
+ * allocating library routine; it needs no nsd_ctx and no plan.
+ *
+ * Same result as nsd_verify_attn(subset = 0) for one layer slab:
+ *   kv_slab     bf16 [num_blocks][2][num_kv_heads][block_size][head_dim] (one layer)
+ *   q, o        bf16 [batch*(gamma+1)][num_q_heads][head_dim]
+ *   h_ctx_len   HOST int32 [batch]  (used to cut the work list; must equal ctx_len)
+ *   ctx_len, kv_indptr, kv_indices   device tables as for nsd_verify_attn
+ * Limits (NSD_ERR_CAPACITY beyond them, nothing launched): batch <= 64;
+ * num_kv_heads <= 8; (num_q_heads/num_kv_heads)*(gamma+1) <= 32; requests longer
+ * than 1024 keys are cut into 1024-key chunks and all such chunks of a call
+ * together must number <= 64 (e.g. eight requests of 8K keys); work items
+ * (chunks of all requests) <= 128.  head_dim 64 or 128, block_size 16
+ * (NSD_ERR_UNSUPPORTED otherwise).  Other errors as nsd_verify_attn.
+ *
+ * The first call on a device resolves the array's address and sets kernel
+ * attributes for that device; make that first call outside any stream capture.
+ * All calls share the one array, and it keeps the previous call's contents: the
+ * call clears the words that must start at zero, but two calls whose kernels can
+ * overlap on the GPU (different streams, or the same call from two threads)
+ * race on the scratch and give undefined results.  Serialise them.  Block ids
+ * that are out of range are replaced by block 0; this variant does not report
+ * them.
+ */
+nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_blocks, int32_t num_q_heads,
+                                  int32_t num_kv_heads, int32_t head_dim, int32_t block_size, const void* q,
+                                  void* o, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
+                                  const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices,
+                                  void* stream);
+
 /* Number of kernels this library has launched through `ctx` since creation. */
 int64_t nsd_launch_count(const nsd_ctx* ctx);
 

@@ -11,5 +11,6 @@ from .api import (  # noqa: F401
     VerifyContext,
     lib_path,
     load_library,
+    nsd_verify_attn_static,
     STATUS,
 )

@@ -82,6 +82,8 @@ def load_library():
     lib.nsd_verify_round.argtypes = [_vp, rap, _vp]
     lib.nsd_verify_round_host.restype = i32
     lib.nsd_verify_round_host.argtypes = [_vp, rap, rap, i64, _vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    lib.nsd_verify_attn_static.restype = i32
+    lib.nsd_verify_attn_static.argtypes = [_vp, i32, i32, i32, i32, i32, _vp, _vp, i32, i32, _vp, _vp, _vp, _vp, _vp]
     lib.nsd_launch_count.restype = i64
     lib.nsd_launch_count.argtypes = [_vp]
     lib.nsd_get_status.restype = i32
@@ -111,6 +113,19 @@ def _stream_handle(stream) -> Optional[int]:
 
         return torch.cuda.current_stream().cuda_stream
     return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def nsd_verify_attn_static(kv_slab, num_blocks, num_q_heads, num_kv_heads, head_dim, block_size, q, o, batch, gamma,
+                           h_ctx_len, ctx_len, kv_indptr, kv_indices, stream=None):
+    """Attention without any device allocation: the scratch is a fixed array inside
+    libnsd.so (see include/nsd.h for who needs this, the size limits and the rule
+    that calls must not overlap on the GPU).  Needs no VerifyContext."""
+    rc = load_library().nsd_verify_attn_static(_ptr(kv_slab), num_blocks, num_q_heads, num_kv_heads, head_dim,
+                                               block_size, _ptr(q), _ptr(o), batch, gamma, _ptr(h_ctx_len),
+                                               _ptr(ctx_len), _ptr(kv_indptr), _ptr(kv_indices),
+                                               _stream_handle(stream))
+    if rc != 0:
+        raise NsdError(rc, "nsd_verify_attn_static")
 
 
 class VerifyContext:

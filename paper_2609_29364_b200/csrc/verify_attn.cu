@@ -29,6 +29,8 @@
 // accumulator.
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "nsd_internal.h"
 
 namespace nsd {
@@ -409,3 +411,129 @@ cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
 }
 
 }  // namespace nsd
+
+// =====================================================================================
+// nsd_verify_attn_static: the same attention kernel for callers that cannot allocate.
+//
+// Some hosts of this library may not call cudaMalloc at all: a plugin running inside
+// another runtime's memory budget, a worker whose device memory was carved up once at
+// start-up (the paper's pre-allocated KV banks are that kind of process), code on a
+// latency path where an allocator call could block on a device-wide synchronisation.
+// For them the split-KV scratch (work list, arrival counters, fp32 partials, status word)
+// lives in the file-scope device array below instead of a caller workspace.  Every GPU
+// that loads the library carries the array until the process exits, so it is kept small
+// and the entry point refuses batches that do not fit.
+// =====================================================================================
+namespace nsd {
+namespace {
+
+constexpr int kStaticMaxBatch = 64;        // requests per call
+constexpr int kStaticMaxSlots = 64;        // chunks of requests that were split (partials kept)
+constexpr int kStaticMaxItems = kStaticMaxBatch + kStaticMaxSlots;
+constexpr int kStaticMaxHkv = 8;
+constexpr int kStaticMaxRows = 32;         // (Hq/Hkv) * (gamma+1)
+constexpr int kStaticMaxD = 128;
+constexpr int kStaticChunkBlocks = 64;     // 1024 keys per chunk
+
+constexpr size_t kStaticOffStatus = 0;
+constexpr size_t kStaticOffCounters = 256;
+constexpr size_t kStaticOffItems = kStaticOffCounters + sizeof(int32_t) * kStaticMaxBatch * kStaticMaxHkv;
+constexpr size_t kStaticOffMl = kStaticOffItems + sizeof(AttnItem) * kStaticMaxItems;
+constexpr size_t kStaticOffAcc = kStaticOffMl + sizeof(float) * 2 * kStaticMaxSlots * kStaticMaxHkv * kStaticMaxRows;
+constexpr size_t kStaticBytes = kStaticOffAcc + sizeof(float) * kStaticMaxSlots * kStaticMaxHkv * kStaticMaxRows * kStaticMaxD;
+static_assert(kStaticOffItems % 256 == 0 && kStaticOffMl % 256 == 0 && kStaticOffAcc % 256 == 0, "scratch sections stay 256-byte aligned");
+static_assert(kStaticBytes <= (9u << 20), "the static scratch is meant to stay modest (about 8.1 MiB)");
+
+// In host code this name is only a handle for cudaGetSymbolAddress; it is NOT a device
+// address and must never be handed to a kernel as a pointer.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_ptr[kMaxDevices];   // device address of the array, per device, set once
+bool g_static_ready[kMaxDevices];
+std::mutex g_static_mutex;
+
+// Once per device, with that device current: resolve the array's device address and opt
+// the kernels in to their shared-memory size.  Neither call allocates.
+cudaError_t static_setup(int device) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_ready[device]) return cudaSuccess;
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (ptr == nullptr) return cudaErrorInvalidSymbol;
+    if ((e = attn_init()) != cudaSuccess) return e;
+    g_static_ptr[device] = static_cast<unsigned char*>(ptr);
+    g_static_ready[device] = true;
+    return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace nsd
+
+extern "C" nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_blocks, int32_t num_q_heads,
+                                             int32_t num_kv_heads, int32_t head_dim, int32_t block_size,
+                                             const void* q, void* o, int32_t batch, int32_t gamma,
+                                             const int32_t* h_ctx_len, const int32_t* ctx_len,
+                                             const int64_t* kv_indptr, const int32_t* kv_indices, void* stream) {
+    using namespace nsd;
+    if (batch < 0 || gamma < 1 || num_blocks < 1 || num_q_heads < 1 || num_kv_heads < 1) return NSD_ERR_INVALID_ARG;
+    if (num_q_heads % num_kv_heads) return NSD_ERR_INVALID_ARG;
+    if ((head_dim != 64 && head_dim != 128) || block_size != kBlockSize) return NSD_ERR_UNSUPPORTED;
+    const int rows = (num_q_heads / num_kv_heads) * (gamma + 1);
+    if (batch > kStaticMaxBatch || num_kv_heads > kStaticMaxHkv || rows > kStaticMaxRows) return NSD_ERR_CAPACITY;
+    if (batch == 0) return NSD_OK;
+    if (!kv_slab || !q || !o || !h_ctx_len || !ctx_len || !kv_indptr || !kv_indices) return NSD_ERR_INVALID_ARG;
+
+    // work list on the stack: requests longer than one chunk are split and keep partials
+    AttnItem items[kStaticMaxItems];
+    int n_items = 0, slots = 0;
+    for (int r = 0; r < batch; ++r) {
+        if (h_ctx_len[r] < 0) return NSD_ERR_INVALID_ARG;
+        const int64_t need = ((int64_t)h_ctx_len[r] + gamma + 1 + kBlockSize - 1) / kBlockSize;
+        const int64_t n = (need + kStaticChunkBlocks - 1) / kStaticChunkBlocks;
+        if (n_items + n > kStaticMaxItems || (n > 1 && slots + n > kStaticMaxSlots)) return NSD_ERR_CAPACITY;
+        for (int c = 0; c < (int)n; ++c) {
+            AttnItem it{};
+            it.req = r;
+            it.blk_begin = c * kStaticChunkBlocks;
+            it.blk_end = (int32_t)(need < (int64_t)(c + 1) * kStaticChunkBlocks ? need : (int64_t)(c + 1) * kStaticChunkBlocks);
+            it.part_base = n > 1 ? slots : -1;
+            it.chunk_idx = c;
+            it.nchunks = (int32_t)n;
+            items[n_items++] = it;
+        }
+        if (n > 1) slots += (int)n;
+    }
+
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return NSD_ERR_CUDA;
+    if (static_setup(device) != cudaSuccess) return NSD_ERR_CUDA;
+    unsigned char* base = g_static_ptr[device];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The array keeps whatever the previous call left: status and counters must start at zero.
+    if (cudaMemsetAsync(base, 0, kStaticOffItems, st) != cudaSuccess) return NSD_ERR_CUDA;
+    // The source is pageable (this stack frame): the runtime has staged it when the call returns.
+    if (cudaMemcpyAsync(base + kStaticOffItems, items, sizeof(AttnItem) * n_items, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return NSD_ERR_CUDA;
+
+    AttnLaunch a{};
+    a.shape = Shape{1, num_blocks, num_q_heads, num_kv_heads, head_dim, block_size};
+    a.pool_slab = static_cast<const uint16_t*>(kv_slab);
+    a.q = static_cast<const uint16_t*>(q);
+    a.o = static_cast<uint16_t*>(o);
+    a.lse = nullptr;
+    a.ctx_len = ctx_len;
+    a.kv_indptr = kv_indptr;
+    a.kv_indices = kv_indices;
+    a.items = reinterpret_cast<const AttnItem*>(base + kStaticOffItems);
+    a.n_items = n_items;
+    a.gamma = gamma;
+    a.part_acc = reinterpret_cast<float*>(base + kStaticOffAcc);
+    a.part_ml = reinterpret_cast<float*>(base + kStaticOffMl);
+    a.counters = reinterpret_cast<int32_t*>(base + kStaticOffCounters);
+    a.status = reinterpret_cast<int32_t*>(base + kStaticOffStatus);
+    a.m_rows = rows;
+    a.tune_stages = 0;
+    return launch_attn(a, st) == cudaSuccess ? NSD_OK : NSD_ERR_CUDA;
+}
