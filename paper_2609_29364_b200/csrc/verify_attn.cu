@@ -70,11 +70,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Byte offset of 16-byte piece `chunk` of row `row` in a swizzled [rows][D] bf16 tile.
+// Shared-memory tiles are [rows][D] bf16 with every row padded by 16 bytes: eight
+// consecutive rows then start 16 bytes apart modulo 128, so the eight row reads of
+// one ldmatrix phase hit distinct banks, and every address used in the main loop is
+// "per-thread constant + compile-time offset" (no swizzle arithmetic per access).
 template <int D>
-__device__ __forceinline__ uint32_t swz(int row, int chunk) {
-    return (uint32_t)(row * (D * 2) + ((chunk ^ (row & 7)) << 4));
-}
+struct Tile {
+    static constexpr int kPitch = D * 2 + 16;                       // bytes per row
+    static constexpr int kBytes = kTileKeys * kPitch;               // K (or V) of one stage
+};
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -84,9 +88,9 @@ __device__ __forceinline__ float ex2_approx(float x) {
 
 template <int D, int kStages>
 struct Smem {
-    static constexpr int kTileBytes = kTileKeys * D * 2;            // K (or V) of one stage
+    static constexpr int kStageBytes = 2 * Tile<D>::kBytes;         // K then V
     static constexpr int kMaxChunkBlocks = 512;
-    static constexpr int kBytes = kStages * 2 * kTileBytes + kMaxChunkBlocks * 4;
+    static constexpr int kBytes = kStages * kStageBytes + kMaxChunkBlocks * 4;
 };
 
 template <int D, int NMT, int kStages>
@@ -96,10 +100,14 @@ verify_attn_kernel(const AttnLaunch a) {
     constexpr int CPR = D / 8;                    // 16-byte pieces per row
     constexpr int KSTEPS = D / 16;                // k-steps of Q K^T
     constexpr int DT = D / 8;                     // n-tiles of P V
-    using SM = Smem<D, kStages>;
+    constexpr int PITCH = Tile<D>::kPitch;
+    constexpr int TILE = Tile<D>::kBytes;
+    constexpr int STAGE = Smem<D, kStages>::kStageBytes;
+    constexpr int ROWS_PER_STEP = NT / CPR;       // rows one pass of all threads covers in a block copy
+    constexpr int COPY_STEPS = (kBlockSize + ROWS_PER_STEP - 1) / ROWS_PER_STEP;
+    static_assert(NT % CPR == 0, "a copy pass covers whole rows");
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* kv_s = smem;
-    int32_t* blk_s = reinterpret_cast<int32_t*>(smem + kStages * 2 * SM::kTileBytes);
+    int32_t* blk_s = reinterpret_cast<int32_t*>(smem + kStages * STAGE);
     __shared__ int s_last;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -128,31 +136,38 @@ verify_attn_kernel(const AttnLaunch a) {
     }
     __syncthreads();                              // blk_s visible before tiles are issued
 
-    const int64_t tile_elems = (int64_t)kBlockSize * D;
-    const uint16_t* k_base = a.pool_slab + (int64_t)head * tile_elems;
-    const uint16_t* v_base = k_base + (int64_t)Hkv * tile_elems;
+    // ---- per-thread constants of the copy and of the fragment loads
+    const uint32_t smem0 = smem_u32(smem);
+    const int cp_row = tid / CPR, cp_ch = tid - cp_row * CPR;
+    const uint32_t cp_dst = smem0 + cp_row * PITCH + cp_ch * 16;               // + stage, K|V, half, step
     const int64_t block_elems = a.shape.block_elems();
+    const uint16_t* k_src = a.pool_slab + (int64_t)head * (kBlockSize * D) + tid * 8;   // + block, step
+    const int64_t v_off = (int64_t)Hkv * (kBlockSize * D);
+    const int mi = lane >> 3;
+    const uint32_t k_frag = smem0 + ((mi >> 1) * 8 + (lane & 7)) * PITCH + (mi & 1) * 16;          // + stage, half, kk
+    const uint32_t v_frag = smem0 + TILE + ((mi & 1) * 8 + (lane & 7)) * PITCH + (mi >> 1) * 16;   // + stage, ks16, dp
 
-    auto issue_tile = [&](int t) {
+    // Issues the copy of tile t (two pool blocks, K and V of this head) into `stage`.
+    auto issue_tile = [&](int t, int stage) {
         if (t < n_tiles) {
-            unsigned char* ks = kv_s + (t % kStages) * 2 * SM::kTileBytes;
-            unsigned char* vs = ks + SM::kTileBytes;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 const int bi = 2 * t + half;
+                const uint32_t dst = cp_dst + stage * STAGE + half * (kBlockSize * PITCH);
                 if (bi < n_blk) {
-                    const int64_t off = (int64_t)blk_s[bi] * block_elems;
-                    for (int c = tid; c < kBlockSize * CPR; c += NT) {
-                        const int row = c / CPR, ch = c - row * CPR;
-                        const uint32_t so = swz<D>(half * kBlockSize + row, ch);
-                        cp_async16(smem_u32(ks) + so, k_base + off + c * 8);
-                        cp_async16(smem_u32(vs) + so, v_base + off + c * 8);
+                    const uint16_t* src = k_src + (int64_t)blk_s[bi] * block_elems;
+#pragma unroll
+                    for (int st = 0; st < COPY_STEPS; ++st) {
+                        if ((st + 1) * ROWS_PER_STEP <= kBlockSize || cp_row + st * ROWS_PER_STEP < kBlockSize) {
+                            cp_async16(dst + st * (ROWS_PER_STEP * PITCH), src + st * (NT * 8));
+                            cp_async16(dst + TILE + st * (ROWS_PER_STEP * PITCH), src + v_off + st * (NT * 8));
+                        }
                     }
                 } else {                           // no such block: V must be finite (zero); K is masked
-                    for (int c = tid; c < kBlockSize * CPR; c += NT) {
-                        const int row = c / CPR, ch = c - row * CPR;
-                        *reinterpret_cast<int4*>(vs + swz<D>(half * kBlockSize + row, ch)) = make_int4(0, 0, 0, 0);
-                    }
+#pragma unroll
+                    for (int st = 0; st < COPY_STEPS; ++st)
+                        if (cp_row + st * ROWS_PER_STEP < kBlockSize)
+                            *reinterpret_cast<int4*>(smem + (dst - smem0) + TILE + st * (ROWS_PER_STEP * PITCH)) = make_int4(0, 0, 0, 0);
                 }
             }
         }
@@ -160,7 +175,7 @@ verify_attn_kernel(const AttnLaunch a) {
     };
 
 #pragma unroll
-    for (int s = 0; s < kStages - 1; ++s) issue_tile(s);
+    for (int s = 0; s < kStages - 1; ++s) issue_tile(s, s);
 
     // ---- per-warp state: rows g and g+8 of m-tile `warp`
     const int g = lane >> 2, tq = lane & 3;
@@ -190,18 +205,19 @@ verify_attn_kernel(const AttnLaunch a) {
     }
 
     const int key0_chunk = it.blk_begin * kBlockSize;
-    for (int t = 0; t < n_tiles; ++t) {
+    // One tile: wait for its copy, refill the stage freed by the previous tile, S = Q K^T,
+    // online softmax, O += P V.  `stage` is a compile-time constant at every call site.
+    auto process_tile = [&](int t, int stage) {
         cp_async_wait<kStages - 2>();
         __syncthreads();
-        issue_tile(t + kStages - 1);
-        unsigned char* ks = kv_s + (t % kStages) * 2 * SM::kTileBytes;
-        unsigned char* vs = ks + SM::kTileBytes;
+        issue_tile(t + kStages - 1, (stage + kStages - 1) % kStages);
         const int key0 = key0_chunk + t * kTileKeys;
         const bool need_mask = key0 + kTileKeys > ctx + 1;   // some key of the tile is hidden from some row
         if (key0 + kTileKeys > n_total) {                    // slots that hold no token: zero their V rows
+            unsigned char* vs = smem + stage * STAGE + TILE;
             for (int c = tid; c < kTileKeys * CPR; c += NT) {
                 const int row = c / CPR, ch = c - row * CPR;
-                if (key0 + row >= n_total) *reinterpret_cast<int4*>(vs + swz<D>(row, ch)) = make_int4(0, 0, 0, 0);
+                if (key0 + row >= n_total) *reinterpret_cast<int4*>(vs + row * PITCH + ch * 16) = make_int4(0, 0, 0, 0);
             }
             __syncthreads();
         }
@@ -212,11 +228,10 @@ verify_attn_kernel(const AttnLaunch a) {
         for (int i = 0; i < 4; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
 #pragma unroll
         for (int kk = 0; kk < KSTEPS; ++kk) {
-            const int mi = lane >> 3;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t kf[4];
-                ldmatrix_x4(kf, smem_u32(ks) + swz<D>(half * 16 + (mi >> 1) * 8 + (lane & 7), kk * 2 + (mi & 1)));
+                ldmatrix_x4(kf, k_frag + stage * STAGE + half * (16 * PITCH) + kk * 32);
                 mma_bf16(s[half * 2 + 0], qf[kk], kf[0], kf[1]);
                 mma_bf16(s[half * 2 + 1], qf[kk], kf[2], kf[3]);
             }
@@ -271,15 +286,20 @@ verify_attn_kernel(const AttnLaunch a) {
         // ---- O += P V
 #pragma unroll
         for (int ks16 = 0; ks16 < 2; ++ks16) {
-            const int mi = lane >> 3;
 #pragma unroll
             for (int dp = 0; dp < DT / 2; ++dp) {
                 uint32_t vf[4];
-                ldmatrix_x4_trans(vf, smem_u32(vs) + swz<D>(ks16 * 16 + (mi & 1) * 8 + (lane & 7), dp * 2 + (mi >> 1)));
+                ldmatrix_x4_trans(vf, v_frag + stage * STAGE + ks16 * (16 * PITCH) + dp * 32);
                 mma_bf16(o_acc[dp * 2 + 0], pf[ks16], vf[0], vf[1]);
                 mma_bf16(o_acc[dp * 2 + 1], pf[ks16], vf[2], vf[3]);
             }
         }
+    };
+
+    for (int t = 0; t < n_tiles; t += kStages) {
+#pragma unroll
+        for (int s = 0; s < kStages; ++s)
+            if (t + s < n_tiles) process_tile(t + s, s);
     }
     cp_async_wait<0>();
 
