@@ -4,29 +4,44 @@
 // spans non-contiguous blocks addressed through a block map).
 //
 // Shape of the work.  For one request and one kv head, the (gamma+1) rows of the
-// G = Hq/Hkv query heads that share the kv head are stacked into one M x D tile
-// (M = G*(gamma+1) = 20 at gamma 4), so every K/V byte is read from HBM once and
-// feeds all M rows through the tensor cores.  The arithmetic intensity is only
-// ~20-36 flop per KV byte, so the kernel is bound by HBM bandwidth; the tensor
-// cores (mma.sync m16n8k16, bf16 in / fp32 accumulate) keep the math off the
-// critical path.
+// G = Hq/Hkv query heads that share the kv head are stacked into M = G*(gamma+1)
+// rows (20 at gamma 4), so every K/V byte is read from HBM once and feeds all M
+// rows.  The arithmetic intensity is only ~20-36 flop per KV byte: the kernel is
+// bound by HBM bandwidth and, under sustained load, by board power, so the design
+// goal is the fewest instructions and shared-memory reads per KV byte.
+//
+// Transposed formulation.  With so few query rows the keys, not the queries, take
+// the 16-wide M dimension of mma.sync.m16n8k16 (bf16 in, fp32 accumulate):
+//     S^T = K  Q^T   A = K tile (16 keys x 16 dims, ldmatrix), B = Q^T held in registers
+//     O^T = V^T P^T  A = V^T tile (16 dims x 16 keys, ldmatrix.trans), B = P^T
+// The query rows are the 8-wide N dimension, so M is padded to a multiple of 8 (24)
+// rather than 16 (32), every K/V fragment is loaded from shared memory once and
+// reused for all row tiles, and one warp serves up to 24 rows.  P^T becomes a B
+// operand by transposing the packed 8x8 accumulator blocks with movmatrix.
 //
 // Parallelisation (split-KV).  The host plan cuts each request's block range into
-// chunks and orders (chunk) items longest first; the grid is one CTA per
-// (item, kv head), scheduled by the hardware in that order.  A CTA has one warp
-// per 16-row m-tile.  K/V tiles of 32 keys stream global -> shared through a
-// cp.async ring (16-byte pieces, XOR-swizzled so ldmatrix is conflict free).
-// Each warp keeps an online softmax (running max / sum in registers, quad
-// shuffles) over its rows.  A request with one chunk writes bf16 output directly;
-// otherwise the CTA stores its unnormalised fp32 partial (max, sum, acc) and the
-// LAST CTA to finish that (request, head) -- decided by an atomic counter, no
-// waiting -- merges all partials in chunk order and writes the output.
+// chunks and orders the chunk items longest first; the grid is one CTA per
+// (item, kv head), scheduled by the hardware in that order.  A CTA has one warp per
+// group of up to three 8-row tiles (one warp at gamma 4).  K/V tiles of one pool block
+// stream global -> shared through a cp.async ring whose rows are padded by 16 bytes
+// (conflict-free ldmatrix, every address a per-thread constant plus a compile-time
+// offset; the ring loop is unrolled by stage).  A request with one chunk writes bf16
+// output directly; otherwise the CTA stores its unnormalised fp32 partial (max, sum,
+// acc) and the LAST CTA to finish that (request, head) -- decided by an atomic
+// counter, nobody waits -- merges all partials in chunk order and writes the output.
 //
-// Masking.  Row i sees keys [0, ctx + i].  Only tiles that reach past ctx need
-// the mask.  Slots past ctx+gamma in the last block may hold anything (NaN
-// included): scores there are replaced by -inf with a select, and the V rows of
-// those slots are zeroed in shared memory, so 0 * NaN never reaches an
-// accumulator.
+// Online softmax.  Each thread keeps the running maximum of its rows in the log2
+// domain with the 1/sqrt(d)*log2(e) scale folded into one FFMA per score.  The
+// running maximum is refreshed (and the accumulators rescaled) only when some score
+// exceeds it by more than 2^8; until then probabilities are simply up to 256 times
+// larger, which fp32 sums and bf16 operands carry without loss, and the common tile
+// needs no cross-lane reduction at all.  Row sums are reduced across lanes once, at
+// the end.
+//
+// Masking.  Row i sees keys [0, ctx + i].  Only tiles that reach past ctx need the
+// mask.  Slots past ctx+gamma in the last block may hold anything (NaN included):
+// scores there are replaced by -inf with a select, and the V rows of those slots are
+// zeroed in shared memory, so 0 * NaN never reaches an accumulator.
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -37,8 +52,8 @@ namespace nsd {
 namespace {
 
 constexpr int kBlockSize = 16;      // keys per pool block
-constexpr int kTileKeys = 32;       // keys per pipeline stage (two pool blocks)
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kMaxSlack = 8.0f;   // the running maximum may lag the true one by this much (log2 units)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -65,49 +80,62 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// Transposes an 8x8 matrix of 16-bit elements held one 32-bit register per lane.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
-
-// Shared-memory tiles are [rows][D] bf16 with every row padded by 16 bytes: eight
-// consecutive rows then start 16 bytes apart modulo 128, so the eight row reads of
-// one ldmatrix phase hit distinct banks, and every address used in the main loop is
-// "per-thread constant + compile-time offset" (no swizzle arithmetic per access).
-template <int D>
-struct Tile {
-    static constexpr int kPitch = D * 2 + 16;                       // bytes per row
-    static constexpr int kBytes = kTileKeys * kPitch;               // K (or V) of one stage
-};
-
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 
-template <int D, int kStages>
-struct Smem {
-    static constexpr int kStageBytes = 2 * Tile<D>::kBytes;         // K then V
-    static constexpr int kMaxChunkBlocks = 512;
-    static constexpr int kBytes = kStages * kStageBytes + kMaxChunkBlocks * 4;
+// Shared-memory tiles are [rows][D] bf16 with every row padded by 16 bytes: eight
+// consecutive rows then start 16 bytes apart modulo 128, so the eight row reads of
+// one ldmatrix phase hit distinct banks.
+template <int D, int TK>
+struct Tile {
+    static constexpr int kPitch = D * 2 + 16;                       // bytes per row
+    static constexpr int kBytes = TK * kPitch;                      // K (or V) of one stage
 };
 
-template <int D, int NMT, int kStages>
-__global__ void __launch_bounds__(NMT * 32)
+// TK = keys per pipeline stage (one or two pool blocks), kStages = ring depth.
+template <int D, int TK, int kStages, int ROWS>
+struct Smem {
+    static constexpr int kStageBytes = 2 * Tile<D, TK>::kBytes;     // K then V
+    static constexpr int kMaxChunkBlocks = 512;
+    static constexpr int kOutPitch = D + 4;                         // floats per staged output row
+    static constexpr int kOutBytes = (ROWS * kOutPitch + 2 * ROWS) * 4;   // output staging reuses the ring
+    static constexpr int kRingBytes = kStages * kStageBytes > kOutBytes ? kStages * kStageBytes : (kOutBytes + 15) / 16 * 16;
+    static constexpr int kBytes = kRingBytes + kMaxChunkBlocks * 4;
+};
+
+// NW warps, each serving NTW tiles of 8 query rows; rows m >= M are zero padding.
+template <int D, int NW, int NTW, int TK, int kStages>
+__global__ void __launch_bounds__(NW * 32)
 verify_attn_kernel(const AttnLaunch a) {
-    constexpr int NT = NMT * 32;                  // threads
+    constexpr int KG = TK / 16;                   // 16-key groups (= pool blocks) per tile
+    constexpr int NT = NW * 32;                   // threads
     constexpr int CPR = D / 8;                    // 16-byte pieces per row
-    constexpr int KSTEPS = D / 16;                // k-steps of Q K^T
-    constexpr int DT = D / 8;                     // n-tiles of P V
-    constexpr int PITCH = Tile<D>::kPitch;
-    constexpr int TILE = Tile<D>::kBytes;
-    constexpr int STAGE = Smem<D, kStages>::kStageBytes;
+    constexpr int KSTEPS = D / 16;                // k-steps of K Q^T
+    constexpr int DM = D / 16;                    // 16-dim m-tiles of V^T P^T
+    constexpr int PITCH = Tile<D, TK>::kPitch;
+    constexpr int TILE = Tile<D, TK>::kBytes;
+    constexpr int ROWS_PAD = NW * NTW * 8;        // query rows incl. padding
+    using SM = Smem<D, TK, kStages, ROWS_PAD>;
+    constexpr int STAGE = SM::kStageBytes;
+    constexpr int OPITCH = SM::kOutPitch;
     constexpr int ROWS_PER_STEP = NT / CPR;       // rows one pass of all threads covers in a block copy
     constexpr int COPY_STEPS = (kBlockSize + ROWS_PER_STEP - 1) / ROWS_PER_STEP;
     static_assert(NT % CPR == 0, "a copy pass covers whole rows");
     extern __shared__ __align__(128) unsigned char smem[];
-    int32_t* blk_s = reinterpret_cast<int32_t*>(smem + kStages * STAGE);
+    int32_t* blk_s = reinterpret_cast<int32_t*>(smem + SM::kRingBytes);
     __shared__ int s_last;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -122,7 +150,7 @@ verify_attn_kernel(const AttnLaunch a) {
     const int M = a.m_rows;
     const int64_t table0 = a.kv_indptr[r];
     const int n_blk = it.blk_end - it.blk_begin;
-    const int n_tiles = (n_blk + 1) >> 1;
+    const int n_tiles = (n_blk + KG - 1) / KG;
 
     // ---- block ids of the chunk -> shared (bad ids are replaced by block 0 and reported)
     for (int i = tid; i < n_blk; i += NT) {
@@ -144,15 +172,18 @@ verify_attn_kernel(const AttnLaunch a) {
     const uint16_t* k_src = a.pool_slab + (int64_t)head * (kBlockSize * D) + tid * 8;   // + block, step
     const int64_t v_off = (int64_t)Hkv * (kBlockSize * D);
     const int mi = lane >> 3;
-    const uint32_t k_frag = smem0 + ((mi >> 1) * 8 + (lane & 7)) * PITCH + (mi & 1) * 16;          // + stage, half, kk
-    const uint32_t v_frag = smem0 + TILE + ((mi & 1) * 8 + (lane & 7)) * PITCH + (mi >> 1) * 16;   // + stage, ks16, dp
+    // K as A operand (16 keys x 16 dims): matrices (keys 0-7|8-15) x (dims 0-7|8-15) -> a0..a3
+    const uint32_t k_frag = smem0 + ((mi & 1) * 8 + (lane & 7)) * PITCH + (mi >> 1) * 16;          // + stage, key group, kk
+    // V^T as A operand (16 dims x 16 keys), read transposed: a0 = keys 0-7 x dims 0-7, a1 = keys 0-7 x dims 8-15,
+    // a2 = keys 8-15 x dims 0-7, a3 = keys 8-15 x dims 8-15
+    const uint32_t v_frag = smem0 + TILE + ((mi >> 1) * 8 + (lane & 7)) * PITCH + (mi & 1) * 16;   // + stage, key group, dm
 
-    // Issues the copy of tile t (two pool blocks, K and V of this head) into `stage`.
+    // Issues the copy of tile t (KG pool blocks, K and V of this head) into `stage`.
     auto issue_tile = [&](int t, int stage) {
         if (t < n_tiles) {
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int bi = 2 * t + half;
+            for (int half = 0; half < KG; ++half) {
+                const int bi = KG * t + half;
                 const uint32_t dst = cp_dst + stage * STAGE + half * (kBlockSize * PITCH);
                 if (bi < n_blk) {
                     const uint16_t* src = k_src + (int64_t)blk_s[bi] * block_elems;
@@ -177,121 +208,145 @@ verify_attn_kernel(const AttnLaunch a) {
 #pragma unroll
     for (int s = 0; s < kStages - 1; ++s) issue_tile(s, s);
 
-    // ---- per-warp state: rows g and g+8 of m-tile `warp`
+    // ---- per-thread view of the fragments: keys g, g+8 of a 16-key group; rows 8j + 2tq + {0,1} of row tile j
     const int g = lane >> 2, tq = lane & 3;
-    const int m_lo = warp * 16 + g, m_hi = m_lo + 8;
-    const int lim_lo = ctx + min(m_lo / G, gamma);      // last visible key of the row
-    const int lim_hi = ctx + min(m_hi / G, gamma);
+    const int row0 = warp * (NTW * 8);                   // first query row of this warp
     const float sc = rsqrtf((float)D) * kLog2e;          // raw score -> log2 domain
-    float o_acc[DT][4];
+    int lim[NTW][2];                                     // last visible key of each of the thread's rows
 #pragma unroll
-    for (int i = 0; i < DT; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
-    float mx_lo = -INFINITY, mx_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-    // ---- Q fragments straight from global memory (row m = i*G + j is query row i of head head*G + j;
-    //      rows past M are zero): a0/a2 = row g, a1/a3 = row g+8, columns kk*16 + {0,8} + 2*tq
-    uint32_t qf[KSTEPS][4];
-    {
-        const uint16_t* q_lo = nullptr;
-        const uint16_t* q_hi = nullptr;
-        if (m_lo < M) q_lo = a.q + (((int64_t)r * (gamma + 1) + m_lo / G) * Hq + head * G + m_lo % G) * D + tq * 2;
-        if (m_hi < M) q_hi = a.q + (((int64_t)r * (gamma + 1) + m_hi / G) * Hq + head * G + m_hi % G) * D + tq * 2;
+    for (int j = 0; j < NTW; ++j)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) lim[j][e] = ctx + min((row0 + j * 8 + tq * 2 + e) / G, gamma);
+
+    // ---- Q^T as B operand, straight from global memory: b0 = (dims 16kk + 2tq, +1; row g), b1 = dims + 8.
+    //      Row m = i*G + h is query row i of head head*G + h; rows past M are zero.
+    uint32_t qb[KSTEPS][NTW][2];
+#pragma unroll
+    for (int j = 0; j < NTW; ++j) {
+        const int m = row0 + j * 8 + g;
+        const uint16_t* qp = nullptr;
+        if (m < M) qp = a.q + (((int64_t)r * (gamma + 1) + m / G) * Hq + head * G + m % G) * D + tq * 2;
 #pragma unroll
         for (int kk = 0; kk < KSTEPS; ++kk) {
-            qf[kk][0] = q_lo ? __ldg(reinterpret_cast<const uint32_t*>(q_lo + kk * 16)) : 0u;
-            qf[kk][1] = q_hi ? __ldg(reinterpret_cast<const uint32_t*>(q_hi + kk * 16)) : 0u;
-            qf[kk][2] = q_lo ? __ldg(reinterpret_cast<const uint32_t*>(q_lo + kk * 16 + 8)) : 0u;
-            qf[kk][3] = q_hi ? __ldg(reinterpret_cast<const uint32_t*>(q_hi + kk * 16 + 8)) : 0u;
+            qb[kk][j][0] = qp ? __ldg(reinterpret_cast<const uint32_t*>(qp + kk * 16)) : 0u;
+            qb[kk][j][1] = qp ? __ldg(reinterpret_cast<const uint32_t*>(qp + kk * 16 + 8)) : 0u;
         }
     }
 
+    float oT[DM][NTW][4];                                // O^T: (dim 16dm + g, rows 2tq,2tq+1), (dim 16dm + g + 8, same rows)
+#pragma unroll
+    for (int dm = 0; dm < DM; ++dm)
+#pragma unroll
+        for (int j = 0; j < NTW; ++j) oT[dm][j][0] = oT[dm][j][1] = oT[dm][j][2] = oT[dm][j][3] = 0.f;
+    float mrun[NTW][2], lsum[NTW][2];                    // running maximum (log2 domain) and this thread's share of the row sum
+#pragma unroll
+    for (int j = 0; j < NTW; ++j) mrun[j][0] = mrun[j][1] = -INFINITY, lsum[j][0] = lsum[j][1] = 0.f;
+
     const int key0_chunk = it.blk_begin * kBlockSize;
-    // One tile: wait for its copy, refill the stage freed by the previous tile, S = Q K^T,
-    // online softmax, O += P V.  `stage` is a compile-time constant at every call site.
+    // One tile: wait for its copy, refill the stage freed by the previous tile, S^T = K Q^T,
+    // online softmax, O^T += V^T P^T.  `stage` is a compile-time constant at every call site.
     auto process_tile = [&](int t, int stage) {
         cp_async_wait<kStages - 2>();
         __syncthreads();
         issue_tile(t + kStages - 1, (stage + kStages - 1) % kStages);
-        const int key0 = key0_chunk + t * kTileKeys;
-        const bool need_mask = key0 + kTileKeys > ctx + 1;   // some key of the tile is hidden from some row
-        if (key0 + kTileKeys > n_total) {                    // slots that hold no token: zero their V rows
+        const int key0 = key0_chunk + t * TK;
+        const bool need_mask = key0 + TK > ctx + 1;   // some key of the tile is hidden from some row
+        if (key0 + TK > n_total) {                    // slots that hold no token: zero their V rows
             unsigned char* vs = smem + stage * STAGE + TILE;
-            for (int c = tid; c < kTileKeys * CPR; c += NT) {
+            for (int c = tid; c < TK * CPR; c += NT) {
                 const int row = c / CPR, ch = c - row * CPR;
                 if (key0 + row >= n_total) *reinterpret_cast<int4*>(vs + row * PITCH + ch * 16) = make_int4(0, 0, 0, 0);
             }
             __syncthreads();
         }
 
-        // ---- S = Q K^T (16 rows x 32 keys per warp)
-        float s[4][4];
+        // ---- S^T = K Q^T: KG groups of 16 keys x NTW row tiles
+        float sT[KG][NTW][4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+        for (int kg = 0; kg < KG; ++kg)
+#pragma unroll
+            for (int j = 0; j < NTW; ++j) sT[kg][j][0] = sT[kg][j][1] = sT[kg][j][2] = sT[kg][j][3] = 0.f;
 #pragma unroll
         for (int kk = 0; kk < KSTEPS; ++kk) {
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
+            for (int kg = 0; kg < KG; ++kg) {
                 uint32_t kf[4];
-                ldmatrix_x4(kf, k_frag + stage * STAGE + half * (16 * PITCH) + kk * 32);
-                mma_bf16(s[half * 2 + 0], qf[kk], kf[0], kf[1]);
-                mma_bf16(s[half * 2 + 1], qf[kk], kf[2], kf[3]);
+                ldmatrix_x4(kf, k_frag + stage * STAGE + kg * (16 * PITCH) + kk * 32);
+#pragma unroll
+                for (int j = 0; j < NTW; ++j) mma_bf16(sT[kg][j], kf, qb[kk][j][0], qb[kk][j][1]);
             }
         }
-        // ---- mask, online softmax (max over raw scores; the scale is folded into the exponent)
-        float tmax_lo = -INFINITY, tmax_hi = -INFINITY;
+        // ---- scale into the log2 domain, mask, thread-local maxima
+        float tmax[NTW][2];
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
+        for (int j = 0; j < NTW; ++j) tmax[j][0] = tmax[j][1] = -INFINITY;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                if (need_mask) {
-                    const int key = key0 + nt * 8 + tq * 2 + e;
-                    s[nt][e] = key <= lim_lo ? s[nt][e] : -INFINITY;
-                    s[nt][2 + e] = key <= lim_hi ? s[nt][2 + e] : -INFINITY;
+        for (int kg = 0; kg < KG; ++kg)
+#pragma unroll
+            for (int j = 0; j < NTW; ++j)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int e = c & 1;
+                    float v = sT[kg][j][c] * sc;
+                    if (need_mask) {
+                        const int key = key0 + kg * 16 + g + (c >> 1) * 8;
+                        v = key <= lim[j][e] ? v : -INFINITY;
+                    }
+                    sT[kg][j][c] = v;
+                    tmax[j][e] = fmaxf(tmax[j][e], v);
                 }
-                tmax_lo = fmaxf(tmax_lo, s[nt][e]);
-                tmax_hi = fmaxf(tmax_hi, s[nt][2 + e]);
+        // ---- refresh the running maxima only when some score outgrows the slack
+        bool outgrown = false;
+#pragma unroll
+        for (int j = 0; j < NTW; ++j)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) outgrown |= tmax[j][e] > mrun[j][e] + kMaxSlack;
+        if (__any_sync(0xffffffffu, outgrown)) {
+#pragma unroll
+            for (int j = 0; j < NTW; ++j)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    float v = tmax[j][e];                 // row maximum over the 8 lanes that share tq
+                    v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 4));
+                    v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 8));
+                    v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 16));
+                    const float m_new = fmaxf(mrun[j][e], v);
+                    // nothing visible yet (m_new = -inf): keep everything at zero without forming inf - inf
+                    const float resc = m_new == -INFINITY ? 1.f : ex2_approx(mrun[j][e] - m_new);
+                    mrun[j][e] = m_new;
+                    lsum[j][e] *= resc;
+#pragma unroll
+                    for (int dm = 0; dm < DM; ++dm) {
+                        oT[dm][j][e] *= resc;
+                        oT[dm][j][2 + e] *= resc;
+                    }
+                }
+        }
+        // ---- P^T = 2^(S^T - m) packed to bf16 and transposed into B fragments
+        uint32_t pb[KG][NTW][2];
+#pragma unroll
+        for (int j = 0; j < NTW; ++j) {
+            const float m0 = mrun[j][0] == -INFINITY ? 0.f : mrun[j][0];
+            const float m1 = mrun[j][1] == -INFINITY ? 0.f : mrun[j][1];
+#pragma unroll
+            for (int kg = 0; kg < KG; ++kg) {
+                const float p0 = ex2_approx(sT[kg][j][0] - m0), p1 = ex2_approx(sT[kg][j][1] - m1);   // key g
+                const float p2 = ex2_approx(sT[kg][j][2] - m0), p3 = ex2_approx(sT[kg][j][3] - m1);   // key g + 8
+                lsum[j][0] += p0 + p2;
+                lsum[j][1] += p1 + p3;
+                pb[kg][j][0] = movmatrix_trans(pack_bf16(p0, p1));
+                pb[kg][j][1] = movmatrix_trans(pack_bf16(p2, p3));
             }
         }
-        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(0xffffffffu, tmax_lo, 1));
-        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(0xffffffffu, tmax_lo, 2));
-        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(0xffffffffu, tmax_hi, 1));
-        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(0xffffffffu, tmax_hi, 2));
-        const float new_lo = fmaxf(mx_lo, tmax_lo), new_hi = fmaxf(mx_hi, tmax_hi);
-        const bool grew = (new_lo != mx_lo) || (new_hi != mx_hi);
-        const float off_lo = new_lo == -INFINITY ? 0.f : -new_lo * sc;   // nothing visible yet: avoid inf - inf
-        const float off_hi = new_hi == -INFINITY ? 0.f : -new_hi * sc;
-        if (__any_sync(0xffffffffu, grew)) {                // rescale only when some row's maximum moved
-            const float resc_lo = ex2_approx(fmaf(mx_lo, sc, off_lo)), resc_hi = ex2_approx(fmaf(mx_hi, sc, off_hi));
-            l_lo *= resc_lo;
-            l_hi *= resc_hi;
+        // ---- O^T += V^T P^T
 #pragma unroll
-            for (int i = 0; i < DT; ++i) {
-                o_acc[i][0] *= resc_lo;
-                o_acc[i][1] *= resc_lo;
-                o_acc[i][2] *= resc_hi;
-                o_acc[i][3] *= resc_hi;
-            }
-        }
-        mx_lo = new_lo;
-        mx_hi = new_hi;
-        uint32_t pf[2][4];                               // P as A-fragments: [k-step of 16 keys]
+        for (int kg = 0; kg < KG; ++kg) {
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
-            const float p0 = ex2_approx(fmaf(s[nt][0], sc, off_lo)), p1 = ex2_approx(fmaf(s[nt][1], sc, off_lo));
-            const float p2 = ex2_approx(fmaf(s[nt][2], sc, off_hi)), p3 = ex2_approx(fmaf(s[nt][3], sc, off_hi));
-            l_lo += p0 + p1;
-            l_hi += p2 + p3;
-            pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
-            pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
-        }
-        // ---- O += P V
-#pragma unroll
-        for (int ks16 = 0; ks16 < 2; ++ks16) {
-#pragma unroll
-            for (int dp = 0; dp < DT / 2; ++dp) {
+            for (int dm = 0; dm < DM; ++dm) {
                 uint32_t vf[4];
-                ldmatrix_x4_trans(vf, v_frag + stage * STAGE + ks16 * (16 * PITCH) + dp * 32);
-                mma_bf16(o_acc[dp * 2 + 0], pf[ks16], vf[0], vf[1]);
-                mma_bf16(o_acc[dp * 2 + 1], pf[ks16], vf[2], vf[3]);
+                ldmatrix_x4_trans(vf, v_frag + stage * STAGE + kg * (16 * PITCH) + dm * 32);
+#pragma unroll
+                for (int j = 0; j < NTW; ++j) mma_bf16(oT[dm][j], vf, pb[kg][j][0], pb[kg][j][1]);
             }
         }
     };
@@ -302,30 +357,56 @@ verify_attn_kernel(const AttnLaunch a) {
             if (t + s < n_tiles) process_tile(t + s, s);
     }
     cp_async_wait<0>();
+    __syncthreads();                                      // the ring is free: reuse it to stage the output
 
-    // ---- row sums across the quad
-    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
-    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
-    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
-    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+    // ---- row sums across the 8 lanes that share tq
+#pragma unroll
+    for (int j = 0; j < NTW; ++j)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            float v = lsum[j][e];
+            v += __shfl_xor_sync(0xffffffffu, v, 4);
+            v += __shfl_xor_sync(0xffffffffu, v, 8);
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
+            lsum[j][e] = v;
+        }
+    // ---- stage O^T as [row][dim] fp32 (+ max, sum per row) so that the stores are row-contiguous
+    float* out_s = reinterpret_cast<float*>(smem);
+    float* ml_s = out_s + ROWS_PAD * OPITCH;              // [row][2]
+#pragma unroll
+    for (int j = 0; j < NTW; ++j)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int m = row0 + j * 8 + tq * 2 + e;
+#pragma unroll
+            for (int dm = 0; dm < DM; ++dm) {
+                out_s[m * OPITCH + dm * 16 + g] = oT[dm][j][e];
+                out_s[m * OPITCH + dm * 16 + g + 8] = oT[dm][j][2 + e];
+            }
+            if (g == 0) {
+                ml_s[m * 2] = mrun[j][e];
+                ml_s[m * 2 + 1] = lsum[j][e];
+            }
+        }
+    __syncthreads();
 
     const int64_t row_base = (int64_t)r * (gamma + 1);
     if (it.part_base < 0) {
-        // ---- single chunk: normalise and write bf16
-#pragma unroll
-        for (int hl = 0; hl < 2; ++hl) {
-            const int m = hl ? m_hi : m_lo;
-            if (m >= M) continue;
-            const float l = hl ? l_hi : l_lo;
-            const float inv = 1.f / l;
-            const int i = m / G, j = m - i * G;
-            const int64_t orow = ((row_base + i) * Hq + head * G + j);
-            uint16_t* op = a.o + orow * D;
-#pragma unroll
-            for (int dt = 0; dt < DT; ++dt)
-                *reinterpret_cast<uint32_t*>(op + dt * 8 + tq * 2) =
-                    pack_bf16(o_acc[dt][hl * 2 + 0] * inv, o_acc[dt][hl * 2 + 1] * inv);
-            if (a.lse && tq == 0) a.lse[orow] = ((hl ? mx_hi : mx_lo) * sc + log2f(l)) * 0.6931471805599453f;
+        // ---- single chunk: normalise and write bf16, 16 bytes per store
+        for (int e = tid; e < M * (D / 8); e += NT) {
+            const int m = e / (D / 8), d8 = e - m * (D / 8);
+            const float inv = 1.f / ml_s[m * 2 + 1];
+            const float4 x = *reinterpret_cast<const float4*>(out_s + m * OPITCH + d8 * 8);
+            const float4 y = *reinterpret_cast<const float4*>(out_s + m * OPITCH + d8 * 8 + 4);
+            const int i = m / G, h = m - i * G;
+            const int64_t orow = (row_base + i) * Hq + head * G + h;
+            uint4 packed;
+            packed.x = pack_bf16(x.x * inv, x.y * inv);
+            packed.y = pack_bf16(x.z * inv, x.w * inv);
+            packed.z = pack_bf16(y.x * inv, y.y * inv);
+            packed.w = pack_bf16(y.z * inv, y.w * inv);
+            *reinterpret_cast<uint4*>(a.o + orow * D + d8 * 8) = packed;
+            if (a.lse && d8 == 0) a.lse[orow] = (ml_s[m * 2] + log2f(ml_s[m * 2 + 1])) * 0.6931471805599453f;
         }
         return;
     }
@@ -335,16 +416,11 @@ verify_attn_kernel(const AttnLaunch a) {
         const int64_t slot = ((int64_t)it.part_base + it.chunk_idx) * Hkv + head;
         float* pa = a.part_acc + slot * M * D;
         float* pm = a.part_ml + slot * M * 2;
-#pragma unroll
-        for (int hl = 0; hl < 2; ++hl) {
-            const int m = hl ? m_hi : m_lo;
-            if (m >= M) continue;
-#pragma unroll
-            for (int dt = 0; dt < DT; ++dt)
-                *reinterpret_cast<float2*>(pa + (int64_t)m * D + dt * 8 + tq * 2) =
-                    make_float2(o_acc[dt][hl * 2 + 0], o_acc[dt][hl * 2 + 1]);
-            if (tq == 0) *reinterpret_cast<float2*>(pm + m * 2) = make_float2((hl ? mx_hi : mx_lo) * sc, hl ? l_hi : l_lo);
+        for (int e = tid; e < M * (D / 4); e += NT) {
+            const int m = e / (D / 4), d4 = e - m * (D / 4);
+            *reinterpret_cast<float4*>(pa + (int64_t)m * D + d4 * 4) = *reinterpret_cast<const float4*>(out_s + m * OPITCH + d4 * 4);
         }
+        for (int e = tid; e < M * 2; e += NT) pm[e] = ml_s[e];
     }
     __threadfence();
     __syncthreads();
@@ -379,8 +455,8 @@ verify_attn_kernel(const AttnLaunch a) {
             l += w * ml.y;
         }
         const float inv = 1.f / l;
-        const int i = m / G, j = m - i * G;
-        const int64_t orow = ((row_base + i) * Hq + head * G + j);
+        const int i = m / G, h = m - i * G;
+        const int64_t orow = ((row_base + i) * Hq + head * G + h);
         uint2 packed;
         packed.x = pack_bf16(acc.x * inv, acc.y * inv);
         packed.y = pack_bf16(acc.z * inv, acc.w * inv);
@@ -389,43 +465,53 @@ verify_attn_kernel(const AttnLaunch a) {
     }
 }
 
-template <int D, int NMT, int kStages>
+template <int D, int NW, int NTW, int TK, int kStages>
 cudaError_t launch_one(const AttnLaunch& a, cudaStream_t stream) {
     const int64_t grid = (int64_t)a.n_items * a.shape.Hkv;
-    verify_attn_kernel<D, NMT, kStages><<<(unsigned)grid, NMT * 32, Smem<D, kStages>::kBytes, stream>>>(a);
+    verify_attn_kernel<D, NW, NTW, TK, kStages><<<(unsigned)grid, NW * 32, Smem<D, TK, kStages, NW * NTW * 8>::kBytes, stream>>>(a);
     return cudaGetLastError();
 }
 
-template <int D, int NMT, int kStages>
+template <int D, int NW, int NTW, int TK, int kStages>
 cudaError_t init_one() {
-    return cudaFuncSetAttribute(verify_attn_kernel<D, NMT, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                Smem<D, kStages>::kBytes);
+    return cudaFuncSetAttribute(verify_attn_kernel<D, NW, NTW, TK, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                Smem<D, TK, kStages, NW * NTW * 8>::kBytes);
 }
 
-constexpr int kStagesD64 = 4, kStagesD128 = 3;
+// One pool block per stage and a deeper ring gave the most resident warps per SM at the same bytes in flight.
+constexpr int kTileKeys = 16, kStagesD64 = 4, kStagesD128 = 4;
+
+// Row tiles of 8: 1..8 of them, spread over warps of at most three tiles each.
+#define NSD_ATTN_SHAPES(X, DD, SS) \
+    X(DD, 1, 1, kTileKeys, SS) X(DD, 1, 2, kTileKeys, SS) X(DD, 1, 3, kTileKeys, SS) X(DD, 2, 2, kTileKeys, SS) X(DD, 2, 3, kTileKeys, SS) X(DD, 3, 3, kTileKeys, SS)
 
 }  // namespace
 
 cudaError_t attn_init() {
     cudaError_t e;
-#define NSD_INIT(DD, NN, SS) \
-    if ((e = init_one<DD, NN, SS>()) != cudaSuccess) return e;
-    NSD_INIT(64, 1, kStagesD64) NSD_INIT(64, 2, kStagesD64) NSD_INIT(64, 3, kStagesD64) NSD_INIT(64, 4, kStagesD64)
-    NSD_INIT(128, 1, kStagesD128) NSD_INIT(128, 2, kStagesD128) NSD_INIT(128, 3, kStagesD128) NSD_INIT(128, 4, kStagesD128)
-    NSD_INIT(128, 2, 2) NSD_INIT(128, 2, 4)
+#define NSD_INIT(DD, WW, TT, KK, SS) \
+    if ((e = init_one<DD, WW, TT, KK, SS>()) != cudaSuccess) return e;
+    NSD_ATTN_SHAPES(NSD_INIT, 64, kStagesD64)
+    NSD_ATTN_SHAPES(NSD_INIT, 128, kStagesD128)
+    NSD_INIT(128, 1, 3, 16, 3) NSD_INIT(128, 1, 3, 32, 2) NSD_INIT(128, 1, 3, 32, 3)
 #undef NSD_INIT
     return cudaSuccess;
 }
 
 cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
     if (a.n_items <= 0) return cudaSuccess;
-    const int nmt = (a.m_rows + 15) / 16;
-    if (a.shape.D == 128 && nmt == 2 && a.tune_stages == 2) return launch_one<128, 2, 2>(a, stream);
-    if (a.shape.D == 128 && nmt == 2 && a.tune_stages == 4) return launch_one<128, 2, 4>(a, stream);
-#define NSD_CASE(DD, NN, SS) \
-    if (a.shape.D == DD && nmt == NN) return launch_one<DD, NN, SS>(a, stream);
-    NSD_CASE(64, 1, kStagesD64) NSD_CASE(64, 2, kStagesD64) NSD_CASE(64, 3, kStagesD64) NSD_CASE(64, 4, kStagesD64)
-    NSD_CASE(128, 1, kStagesD128) NSD_CASE(128, 2, kStagesD128) NSD_CASE(128, 3, kStagesD128) NSD_CASE(128, 4, kStagesD128)
+    const int nt8 = (a.m_rows + 7) / 8;                  // row tiles needed
+    if (nt8 < 1 || nt8 > 8) return cudaErrorInvalidValue;
+    const int nw = (nt8 + 2) / 3, ntw = (nt8 + nw - 1) / nw;
+    if (a.shape.D == 128 && nw == 1 && ntw == 3) {      // experiment knob: tile keys * 10 + ring depth
+        if (a.tune_stages == 163) return launch_one<128, 1, 3, 16, 3>(a, stream);
+        if (a.tune_stages == 322) return launch_one<128, 1, 3, 32, 2>(a, stream);
+        if (a.tune_stages == 323) return launch_one<128, 1, 3, 32, 3>(a, stream);
+    }
+#define NSD_CASE(DD, WW, TT, KK, SS) \
+    if (a.shape.D == DD && nw == WW && ntw == TT) return launch_one<DD, WW, TT, KK, SS>(a, stream);
+    NSD_ATTN_SHAPES(NSD_CASE, 64, kStagesD64)
+    NSD_ATTN_SHAPES(NSD_CASE, 128, kStagesD128)
 #undef NSD_CASE
     return cudaErrorInvalidValue;
 }
