@@ -240,6 +240,7 @@ def run_ours(args):
     import torch.distributed as dist
 
     import paper_2609_29364_b200 as nsd
+    from paper_2609_29364_b200 import dist_util
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -252,7 +253,7 @@ def run_ours(args):
     n_gpus = world
 
     base = pick_config(args)
-    cfg = base if rank == 0 else W.RoundConfig(**{**base.__dict__, "seed": base.seed + 1000 * rank})
+    cfg = dist_util.rank_config(base, rank)          # every rank draws its own batch (weak scaling)
     meta = W.make_batch_meta(cfg)
     host = host_inputs(cfg, meta)
     L, B, g1 = cfg.num_layers, cfg.batch, cfg.gamma + 1
@@ -292,11 +293,7 @@ def run_ours(args):
         torch.cuda.synchronize(device)
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return dist_util.combine(x, 0.0, device)[0]
 
     def timed(fn, steps, warmup):
         """ms per step of fn(), CUDA events on the launching stream, max over ranks."""

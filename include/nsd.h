@@ -67,7 +67,8 @@ typedef enum {
     NSD_ERR_UNSUPPORTED = 4,   /* head_dim / block_size / group size this build has no kernel for */
     NSD_ERR_CUDA = 5,          /* a CUDA runtime call failed; see nsd_last_error             */
     NSD_ERR_DEVICE_FAULT = 6,  /* a kernel met an out-of-range index in a device table       */
-    NSD_ERR_NOT_PLANNED = 7    /* nsd_verify_attn / nsd_verify_round before nsd_verify_plan  */
+    NSD_ERR_NOT_PLANNED = 7,   /* nsd_verify_attn / nsd_verify_round before nsd_verify_plan  */
+    NSD_ERR_TIMEOUT = 8        /* a bounded wait inside a kernel ran out (reported by nsd_get_status) */
 } nsd_status;
 
 typedef struct nsd_ctx nsd_ctx;
@@ -292,7 +293,8 @@ nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_blocks, int32
 int64_t nsd_launch_count(const nsd_ctx* ctx);
 
 /* Synchronises the device work of `ctx` on `stream` and the side stream, then
- * reads the status word: NSD_OK, or NSD_ERR_DEVICE_FAULT with the first
+ * reads the status word: NSD_OK, NSD_ERR_TIMEOUT (a copy never signalled its
+ * barrier within the kernel's bounded wait), or NSD_ERR_DEVICE_FAULT with the first
  * offending request index (or -1) in *first_bad_request (nullable).  The word
  * is cleared by the call. */
 nsd_status nsd_get_status(nsd_ctx* ctx, void* stream, int32_t* first_bad_request);

@@ -14,6 +14,7 @@ _lib = None
 STATUS = {
     0: "NSD_OK", 1: "NSD_ERR_INVALID_ARG", 2: "NSD_ERR_OUT_OF_RANGE", 3: "NSD_ERR_CAPACITY",
     4: "NSD_ERR_UNSUPPORTED", 5: "NSD_ERR_CUDA", 6: "NSD_ERR_DEVICE_FAULT", 7: "NSD_ERR_NOT_PLANNED",
+    8: "NSD_ERR_TIMEOUT",
 }
 
 

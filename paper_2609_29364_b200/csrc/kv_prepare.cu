@@ -4,64 +4,109 @@
 // destination bank is filled before it computes).
 //
 // Both kernels only move bytes.  The gather moves contiguous (slab, block)
-// chunks (64 KiB at the Qwen3-8B shape) with 32-byte accesses that bypass L1 and
-// are marked evict-first, so a copy running beside attention does not push
-// attention's tiles out of L2.
+// chunks (64 KiB at the Qwen3-8B shape) with bulk asynchronous copies
+// (cp.async.bulk, the 1-D TMA path): global -> shared -> global, driven by one
+// thread per CTA, so a copy running beside attention costs the SMs almost no
+// issue slots.
 #include "nsd_internal.h"
 
 namespace nsd {
 namespace {
 
-struct __align__(32) Vec32 {
-    uint32_t w[8];
-};
-// 32-byte accesses (sm_100): no L1 allocation, evict-first in L2.
-__device__ __forceinline__ Vec32 ld_stream(const void* p) {
-    Vec32 v;
-    asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]), "=r"(v.w[7])
-                 : "l"(p));
-    return v;
-}
-__device__ __forceinline__ void st_stream(void* p, const Vec32& v) {
-    asm volatile("st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p),
-                 "r"(v.w[0]), "r"(v.w[1]), "r"(v.w[2]), "r"(v.w[3]), "r"(v.w[4]), "r"(v.w[5]), "r"(v.w[6]), "r"(v.w[7])
-                 : "memory");
-}
+// ---- gather: bulk copies (TMA) ------------------------------------------------------
+// One elected thread per CTA moves kBulkBytes pieces global -> shared -> global with
+// cp.async.bulk, kBulkSlots pieces in flight: the load of a piece completes on an
+// mbarrier (transaction bytes), its store is a bulk group, and a slot is reused once the
+// store has finished READING shared memory.  No other thread touches the data, so the SM
+// spends a handful of instructions per 16 KiB.  Every wait is bounded: on a timeout the
+// CTA records STATUS_TIMEOUT, drains what it can and returns.
+constexpr int kBulkBytes = 16 * 1024;
+constexpr int kBulkSlots = 4;
+constexpr uint32_t kBulkSpinLimit = 1u << 22;
 
-constexpr int kGatherThreads = 256;
-constexpr int kGatherUnroll = 4;                                        // 32-byte accesses in flight per thread
-constexpr int kGatherUnitBytes = kGatherThreads * kGatherUnroll * 32;   // 32 KiB per CTA iteration
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-// One unit = kGatherUnitBytes of one block pair.  block_bytes is a multiple of 32.
-__global__ void __launch_bounds__(kGatherThreads)
-gather_blocks_kernel(uint16_t* __restrict__ slab, int64_t n_pairs, const int32_t* __restrict__ src,
-                     const int32_t* __restrict__ dst, int32_t num_blocks, int64_t block_bytes, int32_t units_per_block,
-                     int32_t* __restrict__ status) {
-    const int64_t n_units = n_pairs * units_per_block;
-    for (int64_t u = blockIdx.x; u < n_units; u += gridDim.x) {
-        const int64_t e = u / units_per_block;
-        const int64_t off = (u - e * units_per_block) * (int64_t)kGatherUnitBytes;
-        const int32_t s = __ldg(src + e), d = __ldg(dst + e);
-        if ((uint32_t)s >= (uint32_t)num_blocks || (uint32_t)d >= (uint32_t)num_blocks) {
-            if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_BLOCK);
-            continue;
-        }
-        const char* sp = reinterpret_cast<const char*>(slab) + (int64_t)s * block_bytes + off;
-        char* dp = reinterpret_cast<char*>(slab) + (int64_t)d * block_bytes + off;
-        const int64_t left = block_bytes - off;                     // bytes of this block still to copy
-        Vec32 v[kGatherUnroll];
-#pragma unroll
-        for (int k = 0; k < kGatherUnroll; ++k) {
-            const int64_t b = ((int64_t)k * kGatherThreads + threadIdx.x) * 32;
-            if (b < left) v[k] = ld_stream(sp + b);
-        }
-#pragma unroll
-        for (int k = 0; k < kGatherUnroll; ++k) {
-            const int64_t b = ((int64_t)k * kGatherThreads + threadIdx.x) * 32;
-            if (b < left) st_stream(dp + b, v[k]);
-        }
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kBulkSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
     }
+    return false;
+}
+
+__global__ void __launch_bounds__(32)
+gather_blocks_bulk_kernel(uint16_t* __restrict__ slab, int64_t n_pairs, const int32_t* __restrict__ src,
+                          const int32_t* __restrict__ dst, int32_t num_blocks, int64_t block_bytes,
+                          int32_t pieces_per_block, int32_t* __restrict__ status) {
+    extern __shared__ __align__(128) unsigned char bulk_smem[];
+    __shared__ __align__(8) uint64_t full_bar[kBulkSlots];
+    if (threadIdx.x != 0) return;                       // a single thread drives the copy engine
+    for (int s = 0; s < kBulkSlots; ++s)
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&full_bar[s])) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+
+    const int64_t n_pieces = n_pairs * pieces_per_block;
+    const int64_t first = blockIdx.x, stride = gridDim.x;
+    const int64_t mine = first < n_pieces ? (n_pieces - first + stride - 1) / stride : 0;
+    auto piece_ptrs = [&](int64_t k, const char*& sp, char*& dp, uint32_t& bytes) -> bool {
+        const int64_t u = first + k * stride;
+        const int64_t e = u / pieces_per_block;
+        const int64_t off = (u - e * pieces_per_block) * (int64_t)kBulkBytes;
+        const int32_t sb = __ldg(src + e), db = __ldg(dst + e);
+        if ((uint32_t)sb >= (uint32_t)num_blocks || (uint32_t)db >= (uint32_t)num_blocks) {
+            atomicOr(status, STATUS_BAD_BLOCK);
+            return false;
+        }
+        sp = reinterpret_cast<const char*>(slab) + (int64_t)sb * block_bytes + off;
+        dp = reinterpret_cast<char*>(slab) + (int64_t)db * block_bytes + off;
+        const int64_t left = block_bytes - off;
+        bytes = (uint32_t)(left < kBulkBytes ? left : kBulkBytes);
+        return true;
+    };
+    auto issue_load = [&](int64_t k) {
+        const int s = (int)(k % kBulkSlots);
+        const char* sp; char* dp; uint32_t bytes;
+        const uint32_t bar = smem_addr(&full_bar[s]);
+        if (!piece_ptrs(k, sp, dp, bytes)) {            // nothing to copy: complete the phase by hand
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+            return;
+        }
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_addr(bulk_smem + s * kBulkBytes)), "l"(sp), "r"(bytes), "r"(bar) : "memory");
+    };
+
+    // Slot reuse: the load of piece k needs the store of piece k - kBulkSlots to have read its data.
+    // Stores are committed one group per piece, in order, so "at most S-1 groups still reading"
+    // with S = kBulkSlots - (lookahead) is the condition; lookahead = kBulkSlots - 1 loads ahead.
+    constexpr int kAhead = kBulkSlots - 1;
+    bool ok = true;
+    for (int64_t k = 0; k < kAhead && k < mine; ++k) issue_load(k);
+    for (int64_t k = 0; k < mine && ok; ++k) {
+        if (k + kAhead < mine) {
+            // slot of piece k + kAhead was last used by piece k - 1: its store must have finished reading
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            issue_load(k + kAhead);
+        }
+        const int s = (int)(k % kBulkSlots);
+        ok = mbar_wait_bounded(smem_addr(&full_bar[s]), (uint32_t)((k / kBulkSlots) & 1));
+        if (!ok) break;
+        const char* sp; char* dp; uint32_t bytes;
+        if (piece_ptrs(k, sp, dp, bytes)) {
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                         ::"l"(dp), "r"(smem_addr(bulk_smem + s * kBulkBytes)), "r"(bytes) : "memory");
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    if (!ok) atomicOr(status, STATUS_TIMEOUT);
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores complete before the CTA retires
 }
 
 // One warp per (row, K|V): copies the Hkv head vectors of one new token into its slot.
@@ -105,16 +150,20 @@ append_tokens_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32
 
 }  // namespace
 
+cudaError_t gather_init() {
+    return cudaFuncSetAttribute(gather_blocks_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBulkSlots * kBulkBytes);
+}
+
 cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const int32_t* src, const int32_t* dst,
                           int32_t* status, cudaStream_t stream) {
     if (n_pairs <= 0) return cudaSuccess;
     const int64_t block_bytes = s.block_elems() * 2;
-    const int32_t upb = (int32_t)((block_bytes + kGatherUnitBytes - 1) / kGatherUnitBytes);
-    const int64_t n_units = n_pairs * upb;
-    // A bounded number of CTAs: the copy shares the SMs with attention.
-    const int64_t max_ctas = 148 * 4;
-    const int grid = (int)(n_units < max_ctas ? n_units : max_ctas);
-    gather_blocks_kernel<<<grid, kGatherThreads, 0, stream>>>(slab, n_pairs, src, dst, s.num_blocks, block_bytes, upb, status);
+    const int32_t ppb = (int32_t)((block_bytes + kBulkBytes - 1) / kBulkBytes);
+    const int64_t n_pieces = n_pairs * ppb;
+    // A bounded number of CTAs (4 per SM, each with 48 KiB of loads in flight): the copy shares the SMs with attention.
+    const int64_t ctas = 148LL * 4;
+    const int grid = (int)(n_pieces < ctas ? n_pieces : ctas);
+    gather_blocks_bulk_kernel<<<grid, 32, kBulkSlots * kBulkBytes, stream>>>(slab, n_pairs, src, dst, s.num_blocks, block_bytes, ppb, status);
     return cudaGetLastError();
 }
 

@@ -114,6 +114,7 @@ const char* nsd_status_string(nsd_status s) {
         case NSD_ERR_CUDA: return "CUDA runtime error";
         case NSD_ERR_DEVICE_FAULT: return "out-of-range index met on the device";
         case NSD_ERR_NOT_PLANNED: return "no plan for this batch";
+        case NSD_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     }
     return "unknown";
 }
@@ -186,6 +187,7 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
         if ((e = cudaEventCreateWithFlags(&ctx->ev_attn[l], cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     }
     if ((e = attn_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(attention)");
+    if ((e = gather_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(gather)");
     *out = ctx;
     return NSD_OK;
 }
@@ -535,6 +537,7 @@ nsd_status nsd_get_status(nsd_ctx* ctx, void* stream, int32_t* first_bad_request
     NSD_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, 4 * sizeof(int32_t), st));
     NSD_CUDA(ctx, cudaStreamSynchronize(st));
     if (first_bad_request) *first_bad_request = ctx->h_status[1] - 1;
+    if (ctx->h_status[0] & STATUS_TIMEOUT) return NSD_ERR_TIMEOUT;
     return ctx->h_status[0] ? NSD_ERR_DEVICE_FAULT : NSD_OK;
 }
 

@@ -20,7 +20,7 @@ struct __align__(16) AttnItem {
 };
 
 // Device status word: [0] = error bits, [1] = first offending request (+1; 0 = none).
-enum : int32_t { STATUS_BAD_BLOCK = 1, STATUS_BAD_TOKEN = 2 };
+enum : int32_t { STATUS_BAD_BLOCK = 1, STATUS_BAD_TOKEN = 2, STATUS_TIMEOUT = 4 };
 
 struct Shape {
     int32_t num_slabs, num_blocks, Hq, Hkv, D, bs;
@@ -56,6 +56,7 @@ cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t
                           const uint16_t* v_new, const uint8_t* is_migrated, int32_t subset, int32_t* status,
                           cudaStream_t stream);
 cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream);
+cudaError_t gather_init();        // opt in to the copy ring's dynamic shared memory, once per device
 cudaError_t attn_init();          // opt in to large dynamic shared memory, once per process
 cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
                           const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int32_t* ctx_len,
