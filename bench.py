@@ -33,6 +33,10 @@ import workload as W  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic byte of verify_attn_kernel, from the
+# ncu capture of the reduced case summarised in profiles/verify_attn_kernel_ncu.md (754.8 MB over 698.9 MB); the
+# full-size launch is too large to capture under the profiler, and traffic grows with the keys streamed.
+ATTN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.080
 
 
 def parse_args():
@@ -426,7 +430,9 @@ def run_ours(args):
             "roofline": {"kernel": "verify_attn_kernel (one launch per layer, timed alone)", "bound": "hbm",
                          "achieved": attn_gbs, "peak": peak, "peak_kind": f"{peak_kind} copy bandwidth",
                          "unit": "GB/s", "frac": attn_gbs / peak, "frac_of_nominal_8TBs": attn_gbs / NOMINAL_HBM_GBS,
-                         "traffic": None, "bytes_per_launch": bytes_["attn_per_layer"], "ms_per_launch": ms_attn_launch},
+                         "traffic": int(ATTN_TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_["attn_per_layer"]),
+                         "traffic_source": "ncu capture of a smaller case scaled by algorithmic bytes (profiles/verify_attn_kernel_ncu.md)",
+                         "bytes_per_launch": bytes_["attn_per_layer"], "ms_per_launch": ms_attn_launch},
             "round_roofline": {"bound": "hbm", "achieved": round_gbs, "peak": peak, "unit": "GB/s",
                                "frac": round_gbs / peak, "frac_of_nominal_8TBs": round_gbs / NOMINAL_HBM_GBS,
                                "algorithmic_bytes_per_round": bytes_["round"]},
