@@ -116,7 +116,7 @@ nsd_status nsd_destroy(nsd_ctx* ctx);
  *                             cover ceil((ctx_len[r]+gamma+1)/block_size)
  *   h_is_migrated  [batch]    nullable; 1 = reassigned to this worker this
  *                             round (its KV arrives through the gather)
- *   chunk_blocks   0 = choose; else the split-KV chunk length in blocks (even)
+ *   chunk_blocks   0 = choose; else the split-KV chunk length in blocks (even, <= 256)
  * Errors: INVALID_ARG (null, negative length, short table), OUT_OF_RANGE
  * (batch > max_batch, gamma outside [1,max_gamma]), CAPACITY (table entries or
  * split count beyond the workspace).  batch == 0 is a valid empty plan.
@@ -217,6 +217,8 @@ typedef struct {
     int32_t* acc_len;
     int32_t* out_tok;
     int32_t* new_ctx_len;         /* nullable */
+    int32_t fuse_gather;          /* 0 = side-stream gather (default), 1 = gather-through attention */
+    int32_t reserved;
 } nsd_round_args;
 
 /*
@@ -228,6 +230,15 @@ typedef struct {
  * acceptance follows the last layer.  With num_slabs < num_layers the gather of
  * layer l also waits for attention of layer l - num_slabs.  Needs a plan for
  * this batch.  Returns after enqueue; `stream` carries the completion.
+ *
+ * fuse_gather = 1 selects the gather-through variant (an extension beyond the
+ * side-stream design; same pool bytes and outputs): there is no copy kernel and
+ * no side stream; attention over a reassigned request reads its committed KV
+ * from the SOURCE blocks, takes the new tokens from k_new / v_new, and writes
+ * both into the destination blocks while it streams them, so the gather's read
+ * disappears.  It needs the plan to have been given is_migrated, and mig_src to
+ * list the reassigned requests' source blocks in request order,
+ * ceil(ctx_len/block_size) entries each (INVALID_ARG if the counts disagree).
  */
 nsd_status nsd_verify_round(nsd_ctx* ctx, const nsd_round_args* args, void* stream);
 

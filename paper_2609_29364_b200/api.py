@@ -39,7 +39,7 @@ class RoundArgs(ctypes.Structure):
         ("batch", ctypes.c_int32), ("gamma", ctypes.c_int32), ("ctx_len", _vp), ("kv_indptr", _vp),
         ("kv_indices", _vp), ("is_migrated", _vp), ("k_new", _vp), ("v_new", _vp), ("q", _vp), ("o", _vp),
         ("p", _vp), ("q_draft", _vp), ("draft_tok", _vp), ("u_acc", _vp), ("u_smp", _vp), ("acc_len", _vp),
-        ("out_tok", _vp), ("new_ctx_len", _vp),
+        ("out_tok", _vp), ("new_ctx_len", _vp), ("fuse_gather", ctypes.c_int32), ("reserved", ctypes.c_int32),
     ]
 
 
@@ -206,7 +206,7 @@ class VerifyContext:
         a = RoundArgs()
         for name, _ in RoundArgs._fields_:
             v = kw.pop(name, None)
-            if name in ("n_mig_blocks", "batch", "gamma"):
+            if name in ("n_mig_blocks", "batch", "gamma", "fuse_gather", "reserved"):
                 setattr(a, name, int(v or 0))
             else:
                 setattr(a, name, _ptr(v))

@@ -35,6 +35,7 @@ struct nsd_ctx {
     bool planned;
     int32_t plan_batch, plan_gamma;
     int32_t n_all, n_res, n_mig_items;
+    int64_t plan_src_blocks;   // source blocks of the planned batch's reassigned requests
     // streams / events
     cudaStream_t side;
     cudaEvent_t ev_start, ev_side_done, ev_plan_free;
@@ -211,7 +212,7 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
                            void* stream) {
     if (!ctx) return NSD_ERR_INVALID_ARG;
     if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
-    if (chunk_blocks < 0 || (chunk_blocks & 1) || chunk_blocks > 512) return NSD_ERR_INVALID_ARG;
+    if (chunk_blocks < 0 || (chunk_blocks & 1) || chunk_blocks > 256) return NSD_ERR_INVALID_ARG;
     if (batch > 0 && (!h_ctx_len || !h_kv_indptr)) return NSD_ERR_INVALID_ARG;
     const int bs = ctx->cfg.block_size;
     const int Hkv = ctx->cfg.num_kv_heads;
@@ -234,7 +235,7 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
     if (cb == 0) {
         const int64_t target_items = 148LL * 3 * 6;                    // SMs x resident CTAs x waves
         int64_t want = (total_blocks * Hkv + target_items - 1) / target_items;
-        want = std::min<int64_t>(std::max<int64_t>(want, 16), 512);
+        want = std::min<int64_t>(std::max<int64_t>(want, 16), 256);
         cb = (int)((want + 1) & ~1LL);
     }
     auto count_slots = [&](int c) {
@@ -246,14 +247,19 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
         return slots;
     };
     while (count_slots(cb) > ctx->part_slots) {
-        if (chunk_blocks != 0 || cb >= 512) return NSD_ERR_CAPACITY;
-        cb = std::min(512, cb * 2);
+        if (chunk_blocks != 0 || cb >= 256) return NSD_ERR_CAPACITY;
+        cb = std::min(256, cb * 2);
     }
     // ---- items
     struct Tmp { AttnItem it; int mig; };
     std::vector<Tmp> items;
     int32_t slot = 0;
+    int64_t src_next = 0;                                                // running offset into the gather's pair list
     for (int r = 0; r < batch; ++r) {
+        const bool mig = h_is_migrated && h_is_migrated[r] != 0;
+        const int64_t src_off = mig ? src_next : -1;
+        if (mig) src_next += ((int64_t)h_ctx_len[r] + bs - 1) / bs;
+        if (src_next > INT32_MAX) return NSD_ERR_CAPACITY;
         const int n = (nblk[r] + cb - 1) / cb;
         int per = (nblk[r] + n - 1) / n;
         per = (per + 1) & ~1;                                            // even: tiles are two blocks
@@ -267,6 +273,7 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
             it.part_base = base;
             it.chunk_idx = c;
             it.nchunks = n_eff;
+            it.src_off = (int32_t)src_off;
             items.push_back({it, h_is_migrated ? (h_is_migrated[r] != 0) : 0});
         }
         if (n_eff > 1) slot += n_eff;
@@ -301,6 +308,7 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
     ctx->n_all = n_all;
     ctx->n_res = n_res;
     ctx->n_mig_items = n_all - n_res;
+    ctx->plan_src_blocks = src_next;
     return NSD_OK;
 }
 
@@ -341,10 +349,23 @@ nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
 }
 
 namespace {
+struct FuseArgs {
+    const int32_t* mig_src;
+    const uint16_t* k_new;     // this layer's rows
+    const uint16_t* v_new;
+};
+
 nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* o, float* lse, int32_t gamma,
                         const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices, int32_t layer,
-                        int32_t subset, cudaStream_t st) {
+                        int32_t subset, cudaStream_t st, const FuseArgs* fuse = nullptr) {
     AttnLaunch a{};
+    if (fuse) {
+        a.fuse = 1;
+        a.pool_slab_w = slab_ptr(ctx, const_cast<void*>(kv_pool), layer);
+        a.mig_src = fuse->mig_src;
+        a.k_new = fuse->k_new;
+        a.v_new = fuse->v_new;
+    }
     a.shape = ctx->shape;
     a.pool_slab = slab_ptr(ctx, const_cast<void*>(kv_pool), layer);
     a.q = static_cast<const uint16_t*>(q);
@@ -424,7 +445,10 @@ nsd_status nsd_verify_round(nsd_ctx* ctx, const nsd_round_args* a, void* stream)
     uint16_t* o = static_cast<uint16_t*>(a->o);
 
     const int64_t n_pairs = a->n_mig_blocks;
-    const bool overlap = n_pairs > 0;
+    if (a->fuse_gather != 0 && a->fuse_gather != 1) return NSD_ERR_INVALID_ARG;
+    if (a->fuse_gather && n_pairs != ctx->plan_src_blocks) return NSD_ERR_INVALID_ARG;   // the plan walks the same list
+    const bool fused = a->fuse_gather && n_pairs > 0;
+    const bool overlap = n_pairs > 0 && !fused;
     if (overlap) {
         NSD_CUDA(ctx, cudaEventRecord(ctx->ev_start, st));
         NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_start, 0));
@@ -451,6 +475,16 @@ nsd_status nsd_verify_round(nsd_ctx* ctx, const nsd_round_args* a, void* stream)
                              a->kv_indptr, a->kv_indices, l, 2, st);
             if (s != NSD_OK) return s;
             if (l + S < L) NSD_CUDA(ctx, cudaEventRecord(ctx->ev_attn[l], st));
+        } else if (fused) {
+            // gather-through: only the resident requests are appended by the copy kernels; attention itself
+            // moves the reassigned requests' blocks and new tokens while it streams them
+            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
+                                        k_new + l * kv_layer, v_new + l * kv_layer, a->is_migrated, 1, ctx->d_status, st));
+            ctx->launches++;
+            const FuseArgs f{a->mig_src, k_new + l * kv_layer, v_new + l * kv_layer};
+            nsd_status s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
+                                        a->kv_indptr, a->kv_indices, l, 0, st, &f);
+            if (s != NSD_OK) return s;
         } else {
             NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
                                         k_new + l * kv_layer, v_new + l * kv_layer, nullptr, 0, ctx->d_status, st));
@@ -471,7 +505,7 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
                                  int64_t* d2h_bytes) {
     if (!ctx || !h || !d) return NSD_ERR_INVALID_ARG;
     const int32_t batch = h->batch, gamma = h->gamma;
-    if (batch != d->batch || gamma != d->gamma || h->n_mig_blocks != d->n_mig_blocks) return NSD_ERR_INVALID_ARG;
+    if (batch != d->batch || gamma != d->gamma || h->n_mig_blocks != d->n_mig_blocks || h->fuse_gather != d->fuse_gather) return NSD_ERR_INVALID_ARG;
     if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
     if (total_table_entries < 0 || total_table_entries > ctx->cfg.max_table_entries || h->n_mig_blocks < 0) return NSD_ERR_INVALID_ARG;
     if (batch == 0) return NSD_OK;

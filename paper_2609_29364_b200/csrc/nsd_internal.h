@@ -16,7 +16,8 @@ struct __align__(16) AttnItem {
     int32_t part_base;   // first partial slot of the request, -1 when it has a single chunk
     int32_t chunk_idx;
     int32_t nchunks;
-    int32_t pad0, pad1;
+    int32_t src_off;     // first entry of the request's source blocks in the gather list, -1 = resident
+    int32_t pad1;
 };
 
 // Device status word: [0] = error bits, [1] = first offending request (+1; 0 = none).
@@ -32,6 +33,13 @@ struct Shape {
 struct AttnLaunch {
     Shape shape;
     const uint16_t* pool_slab;   // base of the layer's slab
+    // gather-through mode (fuse != 0): items with src_off >= 0 stream their committed KV from the source
+    // blocks, take the new tokens from k_new / v_new, and write both to the destination blocks as they go
+    int32_t fuse;
+    uint16_t* pool_slab_w;
+    const int32_t* mig_src;
+    const uint16_t* k_new;       // this layer's [rows][Hkv][D]
+    const uint16_t* v_new;
     const uint16_t* q;
     uint16_t* o;
     float* lse;

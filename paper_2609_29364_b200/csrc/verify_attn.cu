@@ -109,11 +109,11 @@ struct Tile {
 template <int D, int TK, int kStages, int ROWS>
 struct Smem {
     static constexpr int kStageBytes = 2 * Tile<D, TK>::kBytes;     // K then V
-    static constexpr int kMaxChunkBlocks = 512;
+    static constexpr int kMaxChunkBlocks = 256;                     // ids to read from + ids to write to
     static constexpr int kOutPitch = D + 4;                         // floats per staged output row
     static constexpr int kOutBytes = (ROWS * kOutPitch + 2 * ROWS) * 4;   // output staging reuses the ring
     static constexpr int kRingBytes = kStages * kStageBytes > kOutBytes ? kStages * kStageBytes : (kOutBytes + 15) / 16 * 16;
-    static constexpr int kBytes = kRingBytes + kMaxChunkBlocks * 4;
+    static constexpr int kBytes = kRingBytes + 2 * kMaxChunkBlocks * 4;
 };
 
 // NW warps, each serving NTW tiles of 8 query rows; rows m >= M are zero padding.
@@ -152,13 +152,32 @@ verify_attn_kernel(const AttnLaunch a) {
     const int n_blk = it.blk_end - it.blk_begin;
     const int n_tiles = (n_blk + KG - 1) / KG;
 
-    // ---- block ids of the chunk -> shared (bad ids are replaced by block 0 and reported)
+    // Gather-through: a reassigned request streams its committed KV from the source blocks and writes it,
+    // with the new tokens, to its destination blocks on the way (uniform per CTA).
+    const bool fused = a.fuse != 0 && it.src_off >= 0;
+    const int n_src = (ctx + kBlockSize - 1) / kBlockSize;       // blocks that hold committed KV
+    int32_t* dst_s = blk_s + SM::kMaxChunkBlocks;
+
+    // ---- block ids of the chunk -> shared (bad ids are replaced by block 0 and reported);
+    //      blk_s = where a tile is read from (-1: nowhere, a fresh block), dst_s = where it is written to
     for (int i = tid; i < n_blk; i += NT) {
         int32_t b = a.kv_indices[table0 + it.blk_begin + i];
         if ((uint32_t)b >= (uint32_t)a.shape.num_blocks) {
             atomicOr(a.status, STATUS_BAD_BLOCK);
             atomicCAS(a.status + 1, 0, r + 1);
             b = 0;
+        }
+        if (fused) {
+            dst_s[i] = b;
+            b = -1;
+            if (it.blk_begin + i < n_src) {
+                b = a.mig_src[(int64_t)it.src_off + it.blk_begin + i];
+                if ((uint32_t)b >= (uint32_t)a.shape.num_blocks) {
+                    atomicOr(a.status, STATUS_BAD_BLOCK);
+                    atomicCAS(a.status + 1, 0, r + 1);
+                    b = 0;
+                }
+            }
         }
         blk_s[i] = b;
     }
@@ -185,7 +204,7 @@ verify_attn_kernel(const AttnLaunch a) {
             for (int half = 0; half < KG; ++half) {
                 const int bi = KG * t + half;
                 const uint32_t dst = cp_dst + stage * STAGE + half * (kBlockSize * PITCH);
-                if (bi < n_blk) {
+                if (bi < n_blk && blk_s[bi] >= 0) {
                     const uint16_t* src = k_src + (int64_t)blk_s[bi] * block_elems;
 #pragma unroll
                     for (int st = 0; st < COPY_STEPS; ++st) {
@@ -194,7 +213,7 @@ verify_attn_kernel(const AttnLaunch a) {
                             cp_async16(dst + TILE + st * (ROWS_PER_STEP * PITCH), src + v_off + st * (NT * 8));
                         }
                     }
-                } else {                           // no such block: V must be finite (zero); K is masked
+                } else {                           // nothing to read: V must be finite (zero); K is masked or injected
 #pragma unroll
                     for (int st = 0; st < COPY_STEPS; ++st)
                         if (cp_row + st * ROWS_PER_STEP < kBlockSize)
@@ -251,6 +270,37 @@ verify_attn_kernel(const AttnLaunch a) {
         issue_tile(t + kStages - 1, (stage + kStages - 1) % kStages);
         const int key0 = key0_chunk + t * TK;
         const bool need_mask = key0 + TK > ctx + 1;   // some key of the tile is hidden from some row
+        if (fused) {
+            unsigned char* ks = smem + stage * STAGE;
+            // new tokens of this request that fall into the tile come from k_new / v_new, not from the pool
+            const int p_lo = max(ctx, key0), p_hi = min(ctx + gamma, key0 + TK - 1);
+            if (p_lo <= p_hi) {
+                const int n_new = p_hi - p_lo + 1;
+                for (int c = tid; c < n_new * 2 * CPR; c += NT) {
+                    const int row = c / (2 * CPR), rem = c - row * (2 * CPR), kv = rem / CPR, ch = rem - kv * CPR;
+                    const int p = p_lo + row;
+                    const uint16_t* nsrc = (kv ? a.v_new : a.k_new) + (((int64_t)r * (gamma + 1) + (p - ctx)) * Hkv + head) * D + ch * 8;
+                    *reinterpret_cast<int4*>(ks + kv * TILE + (p - key0) * PITCH + ch * 16) = __ldg(reinterpret_cast<const int4*>(nsrc));
+                }
+                __syncthreads();
+            }
+            // write the tile to its destination blocks: whole blocks that had a source, else only the new tokens
+#pragma unroll
+            for (int half = 0; half < KG; ++half) {
+                const int bi = KG * t + half;
+                if (bi >= n_blk) continue;
+                const bool whole = blk_s[bi] >= 0;
+                const int r_lo = whole ? 0 : max(ctx - (key0 + half * 16), 0);
+                const int r_hi = whole ? kBlockSize - 1 : min(ctx + gamma - (key0 + half * 16), kBlockSize - 1);
+                uint16_t* dbase = a.pool_slab_w + (int64_t)dst_s[bi] * block_elems + (int64_t)head * (kBlockSize * D);
+                for (int c = tid; c < (r_hi - r_lo + 1) * 2 * CPR; c += NT) {
+                    const int row = r_lo + c / (2 * CPR), rem = c % (2 * CPR), kv = rem / CPR, ch = rem - kv * CPR;
+                    const int4 v = *reinterpret_cast<const int4*>(ks + kv * TILE + (half * 16 + row) * PITCH + ch * 16);
+                    *reinterpret_cast<int4*>(dbase + (int64_t)kv * v_off + row * D + ch * 8) = v;
+                }
+            }
+            __syncthreads();                                  // the copy has read the tile before anything zeroes it
+        }
         if (key0 + TK > n_total) {                    // slots that hold no token: zero their V rows
             unsigned char* vs = smem + stage * STAGE + TILE;
             for (int c = tid; c < TK * CPR; c += NT) {

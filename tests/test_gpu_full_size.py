@@ -35,7 +35,7 @@ def _sample_requests(cfg, meta, n_random=3):
     return np.array(sorted(picks), dtype=np.int32)
 
 
-def _full_round_check(cfg, slabs, layers_to_check, slabs_to_check):
+def _full_round_check(cfg, slabs, layers_to_check, slabs_to_check, fuse=False):
     meta = W.make_batch_meta(cfg)
     L, B, g1 = cfg.num_layers, cfg.batch, cfg.gamma + 1
     base = W.pool_layer(cfg, meta, 0)                       # every slab starts from these bytes (as in the bench)
@@ -55,7 +55,8 @@ def _full_round_check(cfg, slabs, layers_to_check, slabs_to_check):
     args = ctx.round_args(kv_pool=pool, n_mig_blocks=db.n_mig_blocks, mig_src=db.mig_src, mig_dst=db.mig_dst, batch=B,
                           gamma=cfg.gamma, ctx_len=db.ctx_len, kv_indptr=db.kv_indptr, kv_indices=db.kv_indices,
                           is_migrated=db.is_migrated, k_new=dev(k_new), v_new=dev(v_new), q=dev(q), o=o, p=dev(p),
-                          q_draft=dev(qd), draft_tok=dev(tok), u_acc=dev(ua), u_smp=dev(us), acc_len=acc, out_tok=out)
+                          q_draft=dev(qd), draft_tok=dev(tok), u_acc=dev(ua), u_smp=dev(us), acc_len=acc, out_tok=out,
+                          fuse_gather=int(fuse))
     ctx.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, meta.is_migrated, cfg.gamma)
     for _ in range(2):                                       # twice: the round is idempotent, as the bench assumes
         ctx.nsd_verify_round(args)
@@ -99,12 +100,18 @@ def test_knee_b512_full_size():
     _full_round_check(cfg, slabs=3, layers_to_check=[0, 4, 35], slabs_to_check=[0, 2])
 
 
+def test_knee_b512_full_size_gather_through():
+    """The same workload through the gather-through variant of the round."""
+    _full_round_check(W.CONFIGS["knee_b512"], slabs=3, layers_to_check=[0, 5, 35], slabs_to_check=[1, 2], fuse=True)
+
+
 def test_migration_b256():
     """BASELINE configs[3]: gamma 6, contexts 1024..8192, 75% reassigned."""
     cfg = W.CONFIGS["migration_b256"]
     if not FULL:
         cfg = W.RoundConfig(**{**cfg.__dict__, "batch": 32})
     _full_round_check(cfg, slabs=2, layers_to_check=[0, 3, 35], slabs_to_check=[1])
+    _full_round_check(cfg, slabs=2, layers_to_check=[2, 35], slabs_to_check=[0], fuse=True)
 
 
 def test_long_b128():

@@ -24,7 +24,7 @@ def _oracle_round(cfg, meta, pool0, k_new, v_new, q, acc_in):
     return pool, outs, acc, out, new_ctx
 
 
-def _run_round(cfg, slabs, host_variant=False, repeat=1):
+def _run_round(cfg, slabs, host_variant=False, repeat=1, fuse=False):
     meta = W.make_batch_meta(cfg)
     pool0 = np.stack([W.pool_layer(cfg, meta, s) for s in range(slabs)])
     k_new, v_new = stack_layers(cfg, meta, "kv")
@@ -42,7 +42,7 @@ def _run_round(cfg, slabs, host_variant=False, repeat=1):
              draft_tok=dev(tok), u_acc=dev(ua), u_smp=dev(us),
              acc_len=torch.full((B,), -7, dtype=torch.int32, device="cuda:0"),
              out_tok=torch.full((B, g1), -7, dtype=torch.int32, device="cuda:0"),
-             new_ctx_len=torch.full((B,), -7, dtype=torch.int32, device="cuda:0"))
+             new_ctx_len=torch.full((B,), -7, dtype=torch.int32, device="cuda:0"), fuse_gather=int(fuse))
     stream = torch.cuda.Stream()
     if host_variant:
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a.view(np.int16) if a.dtype == np.uint16 else a)).pin_memory()
@@ -53,7 +53,7 @@ def _run_round(cfg, slabs, host_variant=False, repeat=1):
                  o=torch.zeros(q.shape, dtype=torch.int16).pin_memory(), p=pin(p), q_draft=pin(qd), draft_tok=pin(tok),
                  u_acc=pin(ua), u_smp=pin(us), acc_len=torch.zeros(B, dtype=torch.int32).pin_memory(),
                  out_tok=torch.zeros((B, g1), dtype=torch.int32).pin_memory(),
-                 new_ctx_len=torch.zeros(B, dtype=torch.int32).pin_memory())
+                 new_ctx_len=torch.zeros(B, dtype=torch.int32).pin_memory(), fuse_gather=int(fuse))
         # the device copies start as garbage: everything must arrive through the call
         for k in ("ctx_len", "kv_indptr", "kv_indices", "is_migrated", "k_new", "v_new", "q", "p", "q_draft",
                   "draft_tok", "u_acc", "u_smp"):
@@ -113,6 +113,39 @@ def test_round_twice_gives_the_same_state():
 def test_host_buffer_round():
     _run_round(MULTI, 2, host_variant=True)
     _run_round(W.CONFIGS["tiny"], 1, host_variant=True, repeat=2)
+
+
+@pytest.mark.parametrize("cfg,slabs", [(W.CONFIGS["tiny"], 1), (MULTI, 5), (MULTI, 2), (NOMIG, 2), (ALLMIG, 1), (ALLMIG, 3)],
+                         ids=["tiny", "multi", "multi_alias2", "nomig", "allmig_alias1", "allmig"])
+def test_gather_through_round_gives_the_same_pool_and_outputs(cfg, slabs):
+    """fuse_gather = 1: attention moves the reassigned requests' blocks itself; same pool bytes, same outputs."""
+    _run_round(cfg, slabs, fuse=True)
+
+
+def test_gather_through_round_repeated_and_from_host_buffers():
+    _run_round(MULTI, 2, fuse=True, repeat=3)
+    _run_round(MULTI, 2, fuse=True, host_variant=True)
+    ctx = _run_round(MULTI, 5, fuse=True)
+    # per layer: one append (resident requests) and one attention launch; one acceptance
+    assert ctx.nsd_launch_count() == 5 * 2 + 1
+
+
+def test_gather_through_needs_a_matching_plan():
+    import paper_2609_29364_b200 as nsd
+    from nsd_testlib import DeviceBatch, make_context
+
+    meta = W.make_batch_meta(MULTI)
+    ctx = make_context(MULTI, meta, num_slabs=2)
+    db = DeviceBatch(meta)
+    z = torch.zeros(8, dtype=torch.int32, device="cuda:0")
+    ctx.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, None, MULTI.gamma)          # planned without the reassignment flags
+    args = ctx.round_args(kv_pool=z, n_mig_blocks=db.n_mig_blocks, mig_src=db.mig_src, mig_dst=db.mig_dst, batch=MULTI.batch,
+                          gamma=MULTI.gamma, ctx_len=db.ctx_len, kv_indptr=db.kv_indptr, kv_indices=db.kv_indices,
+                          is_migrated=db.is_migrated, k_new=z, v_new=z, q=z, o=z, p=z, q_draft=z, draft_tok=z, u_acc=z,
+                          u_smp=z, acc_len=z, out_tok=z, fuse_gather=1)
+    with pytest.raises(nsd.NsdError) as e:
+        ctx.nsd_verify_round(args)
+    assert e.value.code == 1 and ctx.nsd_launch_count() == 0
 
 
 def test_launch_count_matches_the_choreography():
