@@ -38,7 +38,8 @@ struct nsd_ctx {
     int64_t plan_src_blocks;   // source blocks of the planned batch's reassigned requests
     // streams / events
     cudaStream_t side;
-    cudaEvent_t ev_start, ev_side_done, ev_plan_free;
+    cudaStream_t copy;         // uploads of the acceptance inputs in nsd_verify_round_host
+    cudaEvent_t ev_start, ev_side_done, ev_plan_free, ev_copy_go, ev_accept_in;
     std::vector<cudaEvent_t> ev_prep, ev_attn;
     int64_t launches;
     char err[256];
@@ -162,7 +163,8 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     ctx->h_items = nullptr;
     ctx->h_status = nullptr;
     ctx->side = nullptr;
-    ctx->ev_start = ctx->ev_side_done = ctx->ev_plan_free = nullptr;
+    ctx->copy = nullptr;
+    ctx->ev_start = ctx->ev_side_done = ctx->ev_plan_free = ctx->ev_copy_go = ctx->ev_accept_in = nullptr;
 
     auto fail = [&](cudaError_t e, const char* what) {
         nsd_status s = cuda_fail(ctx, e, what);
@@ -178,6 +180,9 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     if ((e = cudaMallocHost(&ctx->h_items, 2 * (size_t)L.max_items * sizeof(AttnItem))) != cudaSuccess) return fail(e, "cudaMallocHost(items)");
     if ((e = cudaMallocHost(&ctx->h_status, 4 * sizeof(int32_t))) != cudaSuccess) return fail(e, "cudaMallocHost(status)");
     if ((e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking)) != cudaSuccess) return fail(e, "cudaStreamCreate");
+    if ((e = cudaStreamCreateWithFlags(&ctx->copy, cudaStreamNonBlocking)) != cudaSuccess) return fail(e, "cudaStreamCreate");
+    if ((e = cudaEventCreateWithFlags(&ctx->ev_copy_go, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+    if ((e = cudaEventCreateWithFlags(&ctx->ev_accept_in, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     if ((e = cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     if ((e = cudaEventCreateWithFlags(&ctx->ev_side_done, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     if ((e = cudaEventCreateWithFlags(&ctx->ev_plan_free, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
@@ -196,6 +201,9 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
 nsd_status nsd_destroy(nsd_ctx* ctx) {
     if (!ctx) return NSD_OK;
     if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
+    if (ctx->copy) { cudaStreamSynchronize(ctx->copy); cudaStreamDestroy(ctx->copy); }
+    if (ctx->ev_copy_go) cudaEventDestroy(ctx->ev_copy_go);
+    if (ctx->ev_accept_in) cudaEventDestroy(ctx->ev_accept_in);
     for (auto ev : ctx->ev_prep) if (ev) cudaEventDestroy(ev);
     for (auto ev : ctx->ev_attn) if (ev) cudaEventDestroy(ev);
     if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
@@ -423,7 +431,22 @@ nsd_status nsd_spec_accept(nsd_ctx* ctx, const float* p, const float* q, const i
     return NSD_OK;
 }
 
+namespace {
+// What the host-buffer variant slips in between the last layer and the acceptance.
+struct BeforeAccept {
+    void* h_o;                 // read the attention output back as soon as the layers are done
+    size_t o_bytes;
+    cudaEvent_t inputs_ready;  // the acceptance inputs arrive on another stream
+};
+nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const BeforeAccept* hook);
+}  // namespace
+
 nsd_status nsd_verify_round(nsd_ctx* ctx, const nsd_round_args* a, void* stream) {
+    return round_impl(ctx, a, stream, nullptr);
+}
+
+namespace {
+nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const BeforeAccept* hook) {
     if (!ctx || !a) return NSD_ERR_INVALID_ARG;
     const int32_t batch = a->batch, gamma = a->gamma;
     if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
@@ -494,11 +517,16 @@ nsd_status nsd_verify_round(nsd_ctx* ctx, const nsd_round_args* a, void* stream)
             if (s != NSD_OK) return s;
         }
     }
+    if (hook) {
+        NSD_CUDA(ctx, cudaMemcpyAsync(hook->h_o, a->o, hook->o_bytes, cudaMemcpyDeviceToHost, st));
+        NSD_CUDA(ctx, cudaStreamWaitEvent(st, hook->inputs_ready, 0));
+    }
     NSD_CUDA(ctx, launch_accept(a->p, a->q_draft, a->draft_tok, a->u_acc, a->u_smp, batch, gamma, ctx->cfg.vocab_size,
                                 a->ctx_len, a->acc_len, a->out_tok, a->new_ctx_len, ctx->d_status, st));
     ctx->launches++;
     return NSD_OK;
 }
+}  // namespace
 
 nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const nsd_round_args* d,
                                  int64_t total_table_entries, void* stream, int64_t* h2d_bytes,
@@ -514,6 +542,9 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
     const int64_t V = ctx->cfg.vocab_size, rows = (int64_t)batch * (gamma + 1);
     int64_t up = 0, down = 0;
     struct Copy { const void* src; const void* dst; int64_t bytes; };
+    // The first nine feed the layers and go ahead of them on `stream`; the last five feed only the acceptance and
+    // travel on the copy stream while the layers run.
+    constexpr int kLayerInputs = 9;
     const Copy ups[] = {
         {h->ctx_len, d->ctx_len, batch * 4LL},
         {h->kv_indptr, d->kv_indptr, (batch + 1) * 8LL},
@@ -537,15 +568,24 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
     if (!h->o || !d->o || !h->acc_len || !d->acc_len || !h->out_tok || !d->out_tok) return NSD_ERR_INVALID_ARG;
     nsd_status s = nsd_verify_plan(ctx, batch, gamma, h->ctx_len, h->kv_indptr, h->is_migrated, 0, stream);
     if (s != NSD_OK) return s;
+    NSD_CUDA(ctx, cudaEventRecord(ctx->ev_copy_go, st));          // the device buffers are free once prior work is done
+    NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->copy, ctx->ev_copy_go, 0));
+    int idx = 0;
     for (const Copy& c : ups) {
+        cudaStream_t target = idx++ < kLayerInputs ? st : ctx->copy;
         if (c.bytes == 0) continue;
-        NSD_CUDA(ctx, cudaMemcpyAsync(const_cast<void*>(c.dst), c.src, (size_t)c.bytes, cudaMemcpyHostToDevice, st));
+        NSD_CUDA(ctx, cudaMemcpyAsync(const_cast<void*>(c.dst), c.src, (size_t)c.bytes, cudaMemcpyHostToDevice, target));
         up += c.bytes;
     }
-    s = nsd_verify_round(ctx, d, stream);
-    if (s != NSD_OK) return s;
+    NSD_CUDA(ctx, cudaEventRecord(ctx->ev_accept_in, ctx->copy));
+    const BeforeAccept hook{h->o, (size_t)(L * rows * Hq * D * 2), ctx->ev_accept_in};
+    s = round_impl(ctx, d, stream, &hook);
+    if (s != NSD_OK) {
+        cudaStreamSynchronize(ctx->copy);
+        return s;
+    }
+    down += (int64_t)hook.o_bytes;
     const Copy downs[] = {
-        {d->o, h->o, L * rows * Hq * D * 2},
         {d->acc_len, h->acc_len, batch * 4LL},
         {d->out_tok, h->out_tok, rows * 4},
         {d->new_ctx_len, h->new_ctx_len, (d->new_ctx_len && h->new_ctx_len) ? batch * 4LL : 0},
