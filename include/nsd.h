@@ -193,6 +193,28 @@ nsd_status nsd_spec_accept(nsd_ctx* ctx, const float* p, const float* q, const i
                            const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len,
                            void* stream);
 
+/*
+ * Suffix commit after the acceptance (Section 5, "Incremental KV writeback": only
+ * the KV suffix that changed is written back, the persistent prefix stays; cost
+ * model Eq. (9), Delta_Q tokens x bytes per token).  Request r committed its anchor
+ * and acc_len[r] drafts, i.e. positions ctx_len[r] .. ctx_len[r]+acc_len[r]; for
+ * layers [layer_begin, layer_begin+layer_count) each of these positions is copied,
+ * K and V of every kv head, from the block kv_indices names to the block
+ * exp_indices names for the same position (entry index position / block_size, same
+ * slot).  Rejected drafts stay behind.  acc_len is read on the device, so the call
+ * can be enqueued right behind nsd_spec_accept / nsd_verify_round.
+ *   acc_len      int32 [batch], each in [0, gamma] (else reported as DEVICE_FAULT)
+ *   exp_indptr / exp_indices   the export copy's table; entries that cannot hold
+ *                a committed position are never read (may be -1)
+ *   new_ctx_len  nullable int32 [batch]: ctx_len[r] + 1 + acc_len[r]
+ * Errors: INVALID_ARG, OUT_OF_RANGE (batch, gamma, layers); bad block ids are
+ * skipped and reported by nsd_get_status.
+ */
+nsd_status nsd_kv_commit(nsd_ctx* ctx, void* kv_pool, int32_t batch, int32_t gamma, const int32_t* ctx_len,
+                         const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
+                         const int64_t* exp_indptr, const int32_t* exp_indices, int32_t* new_ctx_len,
+                         int32_t layer_begin, int32_t layer_count, void* stream);
+
 /* Per-round tensors of nsd_verify_round; every pointer on the device. */
 typedef struct {
     void* kv_pool;

@@ -37,6 +37,8 @@ def _load():
         lib.oracle_hardware_threads.restype = i32
         lib.oracle_kv_prepare.restype = i32
         lib.oracle_kv_prepare.argtypes = [vp, i32, i64, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i32, i32]
+        lib.oracle_kv_commit.restype = i32
+        lib.oracle_kv_commit.argtypes = [vp, i32, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, i32, i32]
         lib.oracle_verify_attn.restype = i32
         lib.oracle_verify_attn.argtypes = [vp, i32, i64, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, i32, vp, i32, i32]
         lib.oracle_spec_accept.restype = i32
@@ -74,6 +76,21 @@ def kv_prepare(pool, mig_indptr, mig_src, mig_dst, ctx_len, kv_indptr, kv_indice
         _ptr(pool, np.uint16), S, NB, Hkv, bs, D, n_mig, _ptr(mig_indptr, np.int64), _ptr(mig_src, np.int32),
         _ptr(mig_dst, np.int32), batch, gamma, _ptr(ctx_len, np.int32), _ptr(kv_indptr, np.int64),
         _ptr(kv_indices, np.int32), _ptr(k_new, np.uint16), _ptr(v_new, np.uint16), layer_begin, layer_count)
+
+
+def kv_commit(pool, ctx_len, acc_len, kv_indptr, kv_indices, exp_indptr, exp_indices, gamma: int,
+              layer_begin: int = 0, layer_count: Optional[int] = None):
+    """In place on `pool`; returns (rc, new_ctx_len)."""
+    S, NB, two, Hkv, bs, D = pool.shape
+    batch = len(ctx_len)
+    if layer_count is None:
+        layer_count = S - layer_begin
+    new_ctx = np.empty(batch, dtype=np.int32)
+    rc = _load().oracle_kv_commit(_ptr(pool, np.uint16), S, NB, Hkv, bs, D, batch, gamma, _ptr(ctx_len, np.int32),
+                                  _ptr(acc_len, np.int32), _ptr(kv_indptr, np.int64), _ptr(kv_indices, np.int32),
+                                  _ptr(exp_indptr, np.int64), _ptr(exp_indices, np.int32), _ptr(new_ctx, np.int32),
+                                  layer_begin, layer_count)
+    return rc, new_ctx
 
 
 def verify_attn(pool, q, ctx_len, kv_indptr, kv_indices, gamma: int, layer: int = 0,

@@ -14,6 +14,8 @@
 //    block ranges; state must be present in the destination bank before Run,
 //    Eq. (F.3)).  The result is its own definition: whole-block copies from
 //    source to destination ids, then the new tokens written through the table.
+//  * oracle_kv_commit   -- Section 5 "Incremental KV writeback" and Eq. (9): only the
+//    committed suffix of each request moves to the export copy.
 //  * oracle_verify_attn -- Section 1 / Appendix G.2: the target processes the
 //    anchor token plus gamma proposal tokens of each request in one pass; the
 //    attention itself is the textbook softmax(q K^T / sqrt(d)) V, causal among
@@ -128,6 +130,38 @@ int oracle_kv_prepare(uint16_t* pool, int num_slabs, int64_t num_blocks, int Hkv
                 }
             }
     }
+    return rc;
+}
+
+// Suffix commit (Section 5, "Incremental KV writeback": only the KV suffix that is
+// not yet persistent is written back, the prefix stays; cost Delta_Q * b_KV of
+// Eq. (9)).  After acceptance, request r has committed its anchor and acc_len[r]
+// drafts: positions ctx_r .. ctx_r + acc_len[r].  Each of them is copied, every kv
+// head, K and V, from the block its table names to the block the export table names
+// (same position -> same entry index and slot).  Rejected drafts are not copied.
+int oracle_kv_commit(uint16_t* pool, int num_slabs, int64_t num_blocks, int Hkv, int bs, int D, int batch, int gamma,
+                     const int32_t* ctx_len, const int32_t* acc_len, const int64_t* kv_indptr,
+                     const int32_t* kv_indices, const int64_t* exp_indptr, const int32_t* exp_indices,
+                     int32_t* new_ctx_len, int layer_begin, int layer_count) {
+    PoolShape ps{num_blocks, Hkv, bs, D};
+    int rc = 0;
+    for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
+        const int64_t slab = l % num_slabs;
+        for (int r = 0; r < batch; ++r) {
+            if (acc_len[r] < 0 || acc_len[r] > gamma) { rc = -6; continue; }
+            for (int t = 0; t <= acc_len[r]; ++t) {
+                const int64_t pos = static_cast<int64_t>(ctx_len[r]) + t;
+                const int64_t from = kv_indices[kv_indptr[r] + pos / bs], to = exp_indices[exp_indptr[r] + pos / bs];
+                if (from < 0 || from >= num_blocks || to < 0 || to >= num_blocks) { rc = -1; continue; }
+                const int slot = static_cast<int>(pos % bs);
+                for (int kv = 0; kv < 2; ++kv)
+                    for (int h = 0; h < Hkv; ++h)
+                        std::memcpy(pool + ps.at(slab, to, kv, h, slot, 0), pool + ps.at(slab, from, kv, h, slot, 0), D * sizeof(uint16_t));
+            }
+        }
+    }
+    if (new_ctx_len)
+        for (int r = 0; r < batch; ++r) new_ctx_len[r] = ctx_len[r] + 1 + acc_len[r];
     return rc;
 }
 

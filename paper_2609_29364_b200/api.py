@@ -75,6 +75,8 @@ def load_library():
     lib.nsd_verify_plan.argtypes = [_vp, i32, i32, _vp, _vp, _vp, i32, _vp]
     lib.nsd_kv_prepare.restype = i32
     lib.nsd_kv_prepare.argtypes = [_vp, _vp, i64, _vp, _vp, i32, i32, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp]
+    lib.nsd_kv_commit.restype = i32
+    lib.nsd_kv_commit.argtypes = [_vp, _vp, i32, i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, _vp]
     lib.nsd_verify_attn.restype = i32
     lib.nsd_verify_attn.argtypes = [_vp, _vp, _vp, _vp, _vp, i32, i32, _vp, _vp, _vp, i32, i32, _vp]
     lib.nsd_spec_accept.restype = i32
@@ -188,6 +190,15 @@ class VerifyContext:
                                             gamma, _ptr(ctx_len), _ptr(kv_indptr), _ptr(kv_indices), _ptr(k_new),
                                             _ptr(v_new), _ptr(is_migrated), append_subset, layer_begin, layer_count,
                                             _stream_handle(stream)), "nsd_kv_prepare")
+
+    def nsd_kv_commit(self, kv_pool, batch, gamma, ctx_len, acc_len, kv_indptr, kv_indices, exp_indptr, exp_indices,
+                      new_ctx_len=None, layer_begin=0, layer_count=None, stream=None):
+        if layer_count is None:
+            layer_count = self.cfg.num_layers - layer_begin
+        self._check(self.lib.nsd_kv_commit(self._h, _ptr(kv_pool), batch, gamma, _ptr(ctx_len), _ptr(acc_len),
+                                           _ptr(kv_indptr), _ptr(kv_indices), _ptr(exp_indptr), _ptr(exp_indices),
+                                           _ptr(new_ctx_len), layer_begin, layer_count, _stream_handle(stream)),
+                    "nsd_kv_commit")
 
     def nsd_verify_attn(self, kv_pool, q, o, lse, batch, gamma, ctx_len, kv_indptr, kv_indices, layer=0, subset=0,
                         stream=None):

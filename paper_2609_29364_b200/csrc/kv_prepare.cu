@@ -148,6 +148,60 @@ append_tokens_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32
     }
 }
 
+// Suffix commit: one warp per (request, token t <= gamma, K|V); a warp whose token was not
+// committed (t > acc_len[r]) leaves at once.  acc_len is read on the device, so the call
+// needs no host round trip after the acceptance kernel.
+__global__ void __launch_bounds__(256)
+commit_suffix_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32_t gamma,
+                     const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ acc_len,
+                     const int64_t* __restrict__ kv_indptr, const int32_t* __restrict__ kv_indices,
+                     const int64_t* __restrict__ exp_indptr, const int32_t* __restrict__ exp_indices,
+                     int32_t* __restrict__ new_ctx_len, int32_t* __restrict__ status) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t n_rows = (int64_t)batch * (gamma + 1);
+    if (warp >= 2 * n_rows) return;
+    const int kv = (int)(warp & 1);
+    const int64_t row = warp >> 1;
+    const int r = (int)(row / (gamma + 1));
+    const int t = (int)(row - (int64_t)r * (gamma + 1));
+    const int acc = acc_len[r];
+    if ((uint32_t)acc > (uint32_t)gamma) {
+        if (lane == 0 && t == 0 && kv == 0) {
+            atomicOr(status, STATUS_BAD_TOKEN);
+            atomicCAS(status + 1, 0, r + 1);
+        }
+        return;
+    }
+    if (new_ctx_len && t == 0 && kv == 0 && lane == 0) new_ctx_len[r] = ctx_len[r] + 1 + acc;
+    if (t > acc) return;
+    const int64_t pos = (int64_t)ctx_len[r] + t;
+    const int64_t j = pos / sh.bs;
+    const int slot = (int)(pos - j * sh.bs);
+    int32_t from = -1, to = -1;
+    if (ctx_len[r] >= 0 && kv_indptr[r] + j < kv_indptr[r + 1] && exp_indptr[r] + j < exp_indptr[r + 1]) {
+        from = kv_indices[kv_indptr[r] + j];
+        to = exp_indices[exp_indptr[r] + j];
+    }
+    if ((uint32_t)from >= (uint32_t)sh.num_blocks || (uint32_t)to >= (uint32_t)sh.num_blocks) {
+        if (lane == 0) {
+            atomicOr(status, STATUS_BAD_BLOCK);
+            atomicCAS(status + 1, 0, r + 1);
+        }
+        return;
+    }
+    const int64_t in_block = (int64_t)kv * sh.Hkv * sh.tile_elems() + (int64_t)slot * sh.D;
+    const uint16_t* srcb = slab + (int64_t)from * sh.block_elems() + in_block;
+    uint16_t* dstb = slab + (int64_t)to * sh.block_elems() + in_block;
+    const int vec_per_head = sh.D / 8;
+    const int n_vec = sh.Hkv * vec_per_head;
+    for (int i = lane; i < n_vec; i += 32) {
+        const int h = i / vec_per_head, c = i - h * vec_per_head;
+        const int4 v = *(reinterpret_cast<const int4*>(srcb + (int64_t)h * sh.tile_elems()) + c);
+        *(reinterpret_cast<int4*>(dstb + (int64_t)h * sh.tile_elems()) + c) = v;
+    }
+}
+
 }  // namespace
 
 cudaError_t gather_init() {
@@ -176,6 +230,18 @@ cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t
     const int grid = (int)((warps * 32 + 255) / 256);
     append_tokens_kernel<<<grid, 256, 0, stream>>>(slab, s, batch, gamma, ctx_len, kv_indptr, kv_indices, k_new, v_new,
                                                    is_migrated, subset, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_commit(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int32_t* ctx_len,
+                          const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
+                          const int64_t* exp_indptr, const int32_t* exp_indices, int32_t* new_ctx_len, int32_t* status,
+                          cudaStream_t stream) {
+    const int64_t warps = 2LL * batch * (gamma + 1);
+    if (warps <= 0) return cudaSuccess;
+    const int grid = (int)((warps * 32 + 255) / 256);
+    commit_suffix_kernel<<<grid, 256, 0, stream>>>(slab, s, batch, gamma, ctx_len, acc_len, kv_indptr, kv_indices, exp_indptr,
+                                                   exp_indices, new_ctx_len, status);
     return cudaGetLastError();
 }
 

@@ -356,6 +356,26 @@ nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
     return NSD_OK;
 }
 
+nsd_status nsd_kv_commit(nsd_ctx* ctx, void* kv_pool, int32_t batch, int32_t gamma, const int32_t* ctx_len,
+                         const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
+                         const int64_t* exp_indptr, const int32_t* exp_indices, int32_t* new_ctx_len,
+                         int32_t layer_begin, int32_t layer_count, void* stream) {
+    if (!ctx) return NSD_ERR_INVALID_ARG;
+    if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
+    if (layer_count < 0) return NSD_ERR_INVALID_ARG;
+    if (layer_begin < 0 || layer_begin + (int64_t)layer_count > ctx->cfg.num_layers) return NSD_ERR_OUT_OF_RANGE;
+    if (batch == 0 || layer_count == 0) return NSD_OK;
+    if (!kv_pool || !ctx_len || !acc_len || !kv_indptr || !kv_indices || !exp_indptr || !exp_indices) return NSD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
+        NSD_CUDA(ctx, launch_commit(ctx->shape, slab_ptr(ctx, kv_pool, l), batch, gamma, ctx_len, acc_len, kv_indptr,
+                                    kv_indices, exp_indptr, exp_indices, l == layer_begin ? new_ctx_len : nullptr,
+                                    ctx->d_status, st));
+        ctx->launches++;
+    }
+    return NSD_OK;
+}
+
 namespace {
 struct FuseArgs {
     const int32_t* mig_src;

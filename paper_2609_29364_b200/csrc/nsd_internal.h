@@ -63,6 +63,10 @@ cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t
                           const int64_t* kv_indptr, const int32_t* kv_indices, const uint16_t* k_new,
                           const uint16_t* v_new, const uint8_t* is_migrated, int32_t subset, int32_t* status,
                           cudaStream_t stream);
+cudaError_t launch_commit(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int32_t* ctx_len,
+                          const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
+                          const int64_t* exp_indptr, const int32_t* exp_indices, int32_t* new_ctx_len, int32_t* status,
+                          cudaStream_t stream);
 cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream);
 cudaError_t gather_init();        // opt in to the copy ring's dynamic shared memory, once per device
 cudaError_t attn_init();          // opt in to large dynamic shared memory, once per process

@@ -239,6 +239,30 @@ def pool_layer(cfg: RoundConfig, meta: BatchMeta, layer: int, poison: bool = Tru
     return pool
 
 
+def export_tables(cfg: RoundConfig, meta: BatchMeta):
+    """Block table of the export copy (the other region) for the suffix commit: same
+    indexing as `kv_indices` (entry j covers positions 16j..16j+15), but only the
+    entries that can hold this round's tokens (positions ctx..ctx+gamma) name a block,
+    drawn from the free blocks of region B; the persistent prefix is -1."""
+    bs = cfg.block_size
+    used = np.zeros(meta.num_blocks, dtype=bool)
+    used[meta.kv_indices] = True
+    used[:meta.region_b_begin] = True
+    free = np.nonzero(~used)[0].astype(np.int32)
+    free = free[_rng(cfg.seed, "blocks_a", 7).permutation(len(free))]
+    exp = np.full(len(meta.kv_indices), -1, dtype=np.int32)
+    need = int(((meta.ctx_len.astype(np.int64) + cfg.gamma) // bs - meta.ctx_len.astype(np.int64) // bs + 1).sum())
+    if need > len(free):
+        raise ValueError(f"export table needs {need} free region-B blocks, the pool has {len(free)} (raise pool_factor)")
+    nxt = 0
+    for r in range(cfg.batch):
+        ctx = int(meta.ctx_len[r])
+        for j in range(ctx // bs, (ctx + cfg.gamma) // bs + 1):
+            exp[meta.kv_indptr[r] + j] = free[nxt]
+            nxt += 1
+    return meta.kv_indptr.copy(), exp
+
+
 def new_kv(cfg: RoundConfig, meta: BatchMeta, layer: int):
     """K and V of the gamma+1 tokens each request verifies this round
     (anchor + drafts), bf16 bits, each [batch*(gamma+1)][num_kv_heads][head_dim]."""
