@@ -325,6 +325,42 @@ nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_blocks, int32
                                   const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices,
                                   void* stream);
 
+/*
+ * Worker-triggered batch reconstruction on the host (Algorithm 1): which requests of
+ * the stage's shared pool the triggered worker verifies next.  All times are seconds
+ * on one clock.  For candidate r:
+ *   S({r}) = max(worker_avail, pred_done[r], kv_ready[r])                    Eq. (6)
+ *   d_r    = max(pred_done[r] + target_interval, S({r})) + slack             Eq. (7)
+ * and a batch B is admissible (Eq. (8)) iff |B| <= max_batch, it fits the worker
+ * (sum of rows / KV blocks / tokens within the capacities, Appendix F.2; a request
+ * that does not fit alone is dropped), and S(B) = max over B of S({r}) <= min over B
+ * of d_r.  Line 1 filters by `eligible`; line 2 ranks -- the paper names the criteria
+ * (predecessor readiness, waiting time, temporal compatibility) but not the key:
+ * this library sorts by d_r, then pred_done (older output first: the aging term),
+ * then S({r}), then index; line 3 keeps the first max_batch; lines 4-8 admit greedily
+ * in that order.  Freezing, PREPARE and RUN are the caller's (nsd_verify_plan and
+ * nsd_verify_round take the chosen batch).
+ *   eligible   nullable uint8 [n] (null = all); pred_done, kv_ready  double [n]
+ *   rows / blocks / tokens   nullable int32 [n] (null = 1 row, 0 blocks, 0 tokens each)
+ *   batch_out  int32 [min(n, max_batch)]: indices of the admitted requests in rank order
+ *   batch_size, batch_start (nullable): |B| and S(B) (worker_avail for an empty batch)
+ * Everything is host memory; nothing is launched.  Errors: INVALID_ARG.
+ */
+typedef struct {
+    double worker_avail;      /* predicted availability of the triggered worker, a_w     */
+    double target_interval;   /* g_s                                                     */
+    double slack;             /* Delta_s                                                 */
+    int32_t max_batch;        /* B_max                                                   */
+    int32_t row_capacity;     /* batch rows the standby bank can take                    */
+    int64_t block_capacity;   /* KV blocks it can take                                   */
+    int64_t token_limit;      /* stage-specific token limit                              */
+} nsd_sched_params;
+
+nsd_status nsd_schedule_batch(const nsd_sched_params* prm, int32_t n, const uint8_t* eligible,
+                              const double* pred_done, const double* kv_ready, const int32_t* rows,
+                              const int32_t* blocks, const int32_t* tokens, int32_t* batch_out,
+                              int32_t* batch_size, double* batch_start);
+
 /* Number of kernels this library has launched through `ctx` since creation. */
 int64_t nsd_launch_count(const nsd_ctx* ctx);
 

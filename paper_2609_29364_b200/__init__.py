@@ -11,6 +11,7 @@ from .api import (  # noqa: F401
     VerifyContext,
     lib_path,
     load_library,
+    nsd_schedule_batch,
     nsd_verify_attn_static,
     STATUS,
 )

@@ -33,6 +33,12 @@ class NsdConfig(ctypes.Structure):
 _vp = ctypes.c_void_p
 
 
+class SchedParams(ctypes.Structure):
+    _fields_ = [("worker_avail", ctypes.c_double), ("target_interval", ctypes.c_double), ("slack", ctypes.c_double),
+                ("max_batch", ctypes.c_int32), ("row_capacity", ctypes.c_int32), ("block_capacity", ctypes.c_int64),
+                ("token_limit", ctypes.c_int64)]
+
+
 class RoundArgs(ctypes.Structure):
     _fields_ = [
         ("kv_pool", _vp), ("n_mig_blocks", ctypes.c_int64), ("mig_src", _vp), ("mig_dst", _vp),
@@ -87,6 +93,9 @@ def load_library():
     lib.nsd_verify_round_host.argtypes = [_vp, rap, rap, i64, _vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     lib.nsd_verify_attn_static.restype = i32
     lib.nsd_verify_attn_static.argtypes = [_vp, i32, i32, i32, i32, i32, _vp, _vp, i32, i32, _vp, _vp, _vp, _vp, _vp]
+    lib.nsd_schedule_batch.restype = i32
+    lib.nsd_schedule_batch.argtypes = [ctypes.POINTER(SchedParams), i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                       ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double)]
     lib.nsd_launch_count.restype = i64
     lib.nsd_launch_count.argtypes = [_vp]
     lib.nsd_get_status.restype = i32
@@ -129,6 +138,28 @@ def nsd_verify_attn_static(kv_slab, num_blocks, num_q_heads, num_kv_heads, head_
                                                _stream_handle(stream))
     if rc != 0:
         raise NsdError(rc, "nsd_verify_attn_static")
+
+
+def nsd_schedule_batch(*, worker_avail, target_interval, slack, max_batch, pred_done, kv_ready, eligible=None,
+                       rows=None, blocks=None, tokens=None, row_capacity=2 ** 31 - 1, block_capacity=2 ** 62,
+                       token_limit=2 ** 62):
+    """Algorithm 1 on the host (numpy arrays in, list of admitted indices and predicted start out)."""
+    import numpy as np
+
+    n = len(pred_done)
+    prm = SchedParams(worker_avail, target_interval, slack, max_batch, row_capacity, block_capacity, token_limit)
+    out = np.empty(max(1, min(n, max(max_batch, 0))), dtype=np.int32)
+    m, start = ctypes.c_int32(0), ctypes.c_double(0.0)
+    f64 = lambda a: None if a is None else np.ascontiguousarray(a, dtype=np.float64)
+    i32a = lambda a: None if a is None else np.ascontiguousarray(a, dtype=np.int32)
+    keep = [f64(pred_done), f64(kv_ready), None if eligible is None else np.ascontiguousarray(eligible, dtype=np.uint8),
+            i32a(rows), i32a(blocks), i32a(tokens)]
+    rc = load_library().nsd_schedule_batch(ctypes.byref(prm), n, _ptr(keep[2]), _ptr(keep[0]), _ptr(keep[1]),
+                                           _ptr(keep[3]), _ptr(keep[4]), _ptr(keep[5]), _ptr(out), ctypes.byref(m),
+                                           ctypes.byref(start))
+    if rc != 0:
+        raise NsdError(rc, "nsd_schedule_batch")
+    return out[:m.value].tolist(), start.value
 
 
 class VerifyContext:
