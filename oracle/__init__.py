@@ -43,6 +43,8 @@ def _load():
         lib.oracle_verify_attn.argtypes = [vp, i32, i64, i32, i32, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, i32, vp, i32, i32]
         lib.oracle_spec_accept.restype = i32
         lib.oracle_spec_accept.argtypes = [vp, vp, vp, vp, vp, i32, i32, i64, vp, vp, vp, vp, i32]
+        lib.oracle_spec_accept_logits.restype = i32
+        lib.oracle_spec_accept_logits.argtypes = [vp, ctypes.c_double, vp, vp, vp, vp, i32, i32, i64, vp, vp, vp, vp, vp, i32]
         _lib = lib
     return _lib
 
@@ -128,4 +130,23 @@ def spec_accept(p, q, draft_tok, u_acc, u_smp, ctx_len: Optional[np.ndarray] = N
         _ptr(new_ctx, np.int32), nt)
     if rc != 0:
         raise RuntimeError(f"oracle_spec_accept failed: {rc}")
+    return acc, out, new_ctx
+
+
+def spec_accept_logits(logits, temperature: float, q, draft_tok, u_acc, u_smp, gamma_r: Optional[np.ndarray] = None,
+                       ctx_len: Optional[np.ndarray] = None, nthreads: Optional[int] = None):
+    """logits fp32 [B][gamma+1][V] (widen bf16 first).  temperature 0 = greedy (q, u_acc, u_smp may be None).
+    Returns (acc_len, out_tok, new_ctx_len or None)."""
+    B, g1, V = logits.shape
+    gamma = g1 - 1
+    acc = np.empty(B, dtype=np.int32)
+    out = np.empty((B, gamma + 1), dtype=np.int32)
+    new_ctx = np.empty(B, dtype=np.int32) if ctx_len is not None else None
+    nt = nthreads or hardware_threads()
+    rc = _load().oracle_spec_accept_logits(
+        _ptr(logits, np.float32), float(temperature), _ptr(q, np.float32), _ptr(draft_tok, np.int32),
+        _ptr(u_acc, np.float32), _ptr(u_smp, np.float32), B, gamma, V, _ptr(gamma_r, np.int32), _ptr(ctx_len, np.int32),
+        _ptr(acc, np.int32), _ptr(out, np.int32), _ptr(new_ctx, np.int32), nt)
+    if rc != 0:
+        raise RuntimeError(f"oracle_spec_accept_logits failed: {rc}")
     return acc, out, new_ctx

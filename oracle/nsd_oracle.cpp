@@ -270,4 +270,90 @@ int oracle_spec_accept(const float* p, const float* q, const int32_t* draft_tok,
     return rc;
 }
 
+// Acceptance straight from target logits (the step in front of oracle_spec_accept: the
+// target's softmax with temperature is part of the rule, p_i = softmax(z_i / T)).
+// logits: [batch][gamma+1][V] fp32 (bf16 callers widen exactly).  gamma_r (nullable):
+// drafts actually proposed for request r (<= gamma); its bonus row is row gamma_r.
+//   T > 0  p in double from the logits (max-subtracted, two passes), then exactly the rule
+//          of oracle_spec_accept with every compare, the residual max(0, p - q) and the
+//          sequential CDF in double.
+//   T == 0 greedy verification: the target's token at position i is argmax_k z_i[k]
+//          (smallest index on ties, NaN never wins); draft i is accepted iff it equals
+//          it; the emitted token is the argmax of row n.  No uniforms, no q.
+int oracle_spec_accept_logits(const float* logits, double temperature, const float* q, const int32_t* draft_tok,
+                              const float* u_acc, const float* u_smp, int batch, int gamma, int64_t vocab,
+                              const int32_t* gamma_r, const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok,
+                              int32_t* new_ctx_len, int nthreads) {
+    std::atomic<int> rc{0};
+    parallel_for(batch, nthreads, [&](int64_t r) {
+        const float* zr = logits + r * (gamma + 1) * vocab;
+        const int g = gamma_r ? gamma_r[r] : gamma;
+        int32_t* out = out_tok + r * (gamma + 1);
+        for (int i = 0; i <= gamma; ++i) out[i] = -1;
+        if (g < 0 || g > gamma) { rc = -7; acc_len[r] = 0; return; }
+        auto argmax_row = [&](int i) {
+            const float* z = zr + static_cast<int64_t>(i) * vocab;
+            int64_t best = -1;
+            for (int64_t k = 0; k < vocab; ++k)
+                if (!(z[k] != z[k]) && (best < 0 || z[k] > z[best])) best = k;
+            return best;
+        };
+        int n = g;
+        int64_t y = -1;
+        if (temperature == 0.0) {
+            for (int i = 0; i < g; ++i)
+                if (argmax_row(i) != draft_tok[r * gamma + i]) { n = i; break; }
+            y = argmax_row(n);
+        } else {
+            std::vector<double> prob(vocab), w(vocab);
+            auto softmax_row = [&](int i) {
+                const float* z = zr + static_cast<int64_t>(i) * vocab;
+                double m = -std::numeric_limits<double>::infinity();
+                for (int64_t k = 0; k < vocab; ++k) if (z[k] > m) m = z[k];
+                double sum = 0.0;
+                for (int64_t k = 0; k < vocab; ++k) { prob[k] = std::exp((static_cast<double>(z[k]) - m) / temperature); sum += prob[k]; }
+                for (int64_t k = 0; k < vocab; ++k) prob[k] /= sum;
+            };
+            const float* qr = q + r * gamma * vocab;
+            for (int i = 0; i < g; ++i) {
+                const int32_t x = draft_tok[r * gamma + i];
+                if (x < 0 || x >= vocab) { rc = -5; n = i; break; }
+                softmax_row(i);
+                const double P = prob[x], Q = qr[i * vocab + x];
+                const double ratio = (Q > 0.0) ? P / Q : (P > 0.0 ? 1.0 : 0.0);
+                const double thr = ratio < 1.0 ? ratio : 1.0;
+                if (!(static_cast<double>(u_acc[r * gamma + i]) < thr)) { n = i; break; }
+            }
+            softmax_row(n);
+            double Z = 0.0;
+            if (n < g) {
+                const float* qrow = qr + static_cast<int64_t>(n) * vocab;
+                for (int64_t k = 0; k < vocab; ++k) {
+                    const double d = prob[k] - static_cast<double>(qrow[k]);
+                    w[k] = d > 0.0 ? d : 0.0;
+                    Z += w[k];
+                }
+            }
+            if (n == g || Z == 0.0) {
+                Z = 0.0;
+                for (int64_t k = 0; k < vocab; ++k) { w[k] = prob[k]; Z += w[k]; }
+            }
+            const double t = static_cast<double>(u_smp[r]) * Z;
+            int64_t last_pos = -1;
+            double C = 0.0;
+            for (int64_t k = 0; k < vocab; ++k) {
+                C += w[k];
+                if (w[k] > 0.0) last_pos = k;
+                if (C > t) { y = k; break; }
+            }
+            if (y < 0) y = last_pos;
+        }
+        acc_len[r] = n;
+        for (int i = 0; i < n; ++i) out[i] = draft_tok[r * gamma + i];
+        out[n] = static_cast<int32_t>(y);
+        if (new_ctx_len && ctx_len) new_ctx_len[r] = ctx_len[r] + 1 + n;
+    });
+    return rc;
+}
+
 }  // extern "C"
