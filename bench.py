@@ -372,6 +372,20 @@ def run_ours(args):
 
     ms_prepare_layer = timed(prepare_all_layers, max(2, args.steps // 2), 1) / L
     ms_accept = timed(accept_only, max(5, args.steps), 2)
+
+    # ---- acceptance straight from logits (the softmax fused in); logits = log p, so the decisions are the same
+    logits = torch.log(d["p"])
+    acc2 = torch.zeros_like(d["acc_len"])
+    out2 = torch.zeros_like(d["out_tok"])
+
+    def accept_logits_only():
+        ctx.nsd_spec_accept_logits(logits, 0, 1.0, d["q_draft"], d["draft_tok"], d["u_acc"], d["u_smp"], B, cfg.gamma, cfg.vocab,
+                                   None, d["ctx_len"], acc2, out2, None, stream=stream)
+
+    ms_accept_logits = timed(accept_logits_only, max(5, args.steps), 2)
+    acc2_h = acc2.cpu().numpy()
+    bytes_accept_logits = int((acc2_h + 1).sum()) * cfg.vocab * 4 + int((acc2_h < cfg.gamma).sum()) * cfg.vocab * 4
+    del logits
     nomig = ctx.round_args(**{**d, "n_mig_blocks": 0, "mig_src": None, "mig_dst": None, "is_migrated": None})
     ms_round_nomig = timed(lambda: ctx.nsd_verify_round(nomig, stream=stream), max(2, args.steps // 2), 1)
     exposed_ms = ms_round - ms_round_nomig
@@ -447,7 +461,10 @@ def run_ours(args):
                              "accept_alone": ms_accept, "round_without_reassignment": ms_round_nomig,
                              "exposed_prepare": exposed_ms, "exposed_prepare_bar": gather_bar_ms,
                              "prepare_GBs_alone": (bytes_["gather_per_layer"] + bytes_["append_per_layer"]) / (ms_prepare_layer * 1e-3) / 1e9,
-                             "accept_GBs_alone": bytes_["accept"] / (ms_accept * 1e-3) / 1e9},
+                             "accept_GBs_alone": bytes_["accept"] / (ms_accept * 1e-3) / 1e9,
+                             "accept_from_logits_alone": ms_accept_logits,
+                             "accept_from_logits_GBs": bytes_accept_logits / (ms_accept_logits * 1e-3) / 1e9,
+                             "accept_from_logits_agrees_on": float((acc2_h == acc_len).mean())},
             "gather_through_round": {
                 "what": "nsd_verify_round with fuse_gather=1: attention reads reassigned requests from their source blocks and "
                         "writes the destination blocks itself; no copy kernel, no side stream; same pool bytes and outputs",

@@ -194,6 +194,32 @@ nsd_status nsd_spec_accept(nsd_ctx* ctx, const float* p, const float* q, const i
                            void* stream);
 
 /*
+ * Acceptance straight from the target's logits: the step in front of nsd_spec_accept
+ * (the p of the cited rule is the target's softmax; with a temperature,
+ * p_i = softmax(z_i / T)), fused so that p is never materialised.
+ *   logits        [batch][gamma+1][vocab], logits_dtype 0 = fp32, 1 = bf16
+ *   temperature   > 0: sample as nsd_spec_accept does, with p formed on the fly;
+ *                 0: greedy verification -- draft i is accepted iff it equals
+ *                 argmax_k z_i[k] (smallest index on ties, NaN never wins) and the
+ *                 emitted token is the argmax of row n; q, u_acc, u_smp may be null
+ *   gamma_r       nullable int32 [batch]: drafts actually proposed for request r
+ *                 (0..gamma; tensors stay padded to gamma); its bonus row is row
+ *                 gamma_r[r]; an impossible value is reported and treated as 0
+ *   everything else as nsd_spec_accept.
+ * Only rows 0..n of a request are read (the sweep stops at the first rejection).
+ * Exponentials are fp32 (ex2.approx), sums and compares fp64: against an all-fp64
+ * evaluation a decision can differ only within fp32 rounding of p at a decision or
+ * CDF boundary; greedy mode is exact.  A row needs a finite maximum.
+ * Errors: INVALID_ARG (null, negative or NaN temperature), OUT_OF_RANGE,
+ * UNSUPPORTED (dtype).
+ */
+nsd_status nsd_spec_accept_logits(nsd_ctx* ctx, const void* logits, int32_t logits_dtype, float temperature,
+                                  const float* q, const int32_t* draft_tok, const float* u_acc, const float* u_smp,
+                                  int32_t batch, int32_t gamma, int32_t vocab, const int32_t* gamma_r,
+                                  const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len,
+                                  void* stream);
+
+/*
  * Suffix commit after the acceptance (Section 5, "Incremental KV writeback": only
  * the KV suffix that changed is written back, the persistent prefix stays; cost
  * model Eq. (9), Delta_Q tokens x bytes per token).  Request r committed its anchor

@@ -87,6 +87,8 @@ def load_library():
     lib.nsd_verify_attn.argtypes = [_vp, _vp, _vp, _vp, _vp, i32, i32, _vp, _vp, _vp, i32, i32, _vp]
     lib.nsd_spec_accept.restype = i32
     lib.nsd_spec_accept.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp, _vp, _vp, _vp, _vp]
+    lib.nsd_spec_accept_logits.restype = i32
+    lib.nsd_spec_accept_logits.argtypes = [_vp, _vp, i32, ctypes.c_float, _vp, _vp, _vp, _vp, i32, i32, i32, _vp, _vp, _vp, _vp, _vp, _vp]
     lib.nsd_verify_round.restype = i32
     lib.nsd_verify_round.argtypes = [_vp, rap, _vp]
     lib.nsd_verify_round_host.restype = i32
@@ -242,6 +244,13 @@ class VerifyContext:
         self._check(self.lib.nsd_spec_accept(self._h, _ptr(p), _ptr(q), _ptr(draft_tok), _ptr(u_acc), _ptr(u_smp),
                                              batch, gamma, vocab, _ptr(ctx_len), _ptr(acc_len), _ptr(out_tok),
                                              _ptr(new_ctx_len), _stream_handle(stream)), "nsd_spec_accept")
+
+    def nsd_spec_accept_logits(self, logits, logits_dtype, temperature, q, draft_tok, u_acc, u_smp, batch, gamma, vocab,
+                               gamma_r, ctx_len, acc_len, out_tok, new_ctx_len=None, stream=None):
+        self._check(self.lib.nsd_spec_accept_logits(self._h, _ptr(logits), logits_dtype, float(temperature), _ptr(q),
+                                                    _ptr(draft_tok), _ptr(u_acc), _ptr(u_smp), batch, gamma, vocab,
+                                                    _ptr(gamma_r), _ptr(ctx_len), _ptr(acc_len), _ptr(out_tok),
+                                                    _ptr(new_ctx_len), _stream_handle(stream)), "nsd_spec_accept_logits")
 
     @staticmethod
     def round_args(**kw) -> RoundArgs:

@@ -451,6 +451,26 @@ nsd_status nsd_spec_accept(nsd_ctx* ctx, const float* p, const float* q, const i
     return NSD_OK;
 }
 
+nsd_status nsd_spec_accept_logits(nsd_ctx* ctx, const void* logits, int32_t logits_dtype, float temperature,
+                                  const float* q, const int32_t* draft_tok, const float* u_acc, const float* u_smp,
+                                  int32_t batch, int32_t gamma, int32_t vocab, const int32_t* gamma_r,
+                                  const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len,
+                                  void* stream) {
+    if (!ctx) return NSD_ERR_INVALID_ARG;
+    if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma || vocab < 1) return NSD_ERR_OUT_OF_RANGE;
+    if (logits_dtype != 0 && logits_dtype != 1) return NSD_ERR_UNSUPPORTED;
+    if (!(temperature >= 0.f)) return NSD_ERR_INVALID_ARG;                       // negative or NaN
+    if (batch == 0) return NSD_OK;
+    if (!logits || !draft_tok || !acc_len || !out_tok) return NSD_ERR_INVALID_ARG;
+    if (temperature > 0.f && (!q || !u_acc || !u_smp)) return NSD_ERR_INVALID_ARG;
+    if ((new_ctx_len != nullptr) && !ctx_len) return NSD_ERR_INVALID_ARG;
+    NSD_CUDA(ctx, launch_accept_logits(logits, logits_dtype, temperature, q, draft_tok, u_acc, u_smp, batch, gamma, vocab,
+                                       gamma_r, ctx_len, acc_len, out_tok, new_ctx_len, ctx->d_status,
+                                       static_cast<cudaStream_t>(stream)));
+    ctx->launches++;
+    return NSD_OK;
+}
+
 namespace {
 // What the host-buffer variant slips in between the last layer and the acceptance.
 struct BeforeAccept {

@@ -75,4 +75,10 @@ cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_t
                           int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
                           cudaStream_t stream);
 
+cudaError_t launch_accept_logits(const void* logits, int32_t logits_bf16, float temperature, const float* q,
+                                 const int32_t* draft_tok, const float* u_acc, const float* u_smp, int32_t batch,
+                                 int32_t gamma, int32_t vocab, const int32_t* gamma_r, const int32_t* ctx_len,
+                                 int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
+                                 cudaStream_t stream);
+
 }  // namespace nsd

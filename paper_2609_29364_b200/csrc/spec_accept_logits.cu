@@ -1,0 +1,171 @@
+// Speculative acceptance straight from the target's logits: the softmax with temperature
+// that turns logits into the p of the acceptance rule (Section 1's cited rule: accept
+// while u < min(1, p/q), residual resampling, bonus token) is fused into the kernel, so
+// the [batch][gamma+1][vocab] probability tensor is never written or re-read.
+//
+// One CTA per request.  Rows are swept in order and only as far as needed: row i costs
+// one pass (block-wide max and sum of exponentials, kept online per thread and merged
+// through shared memory), after which warp 0 can test draft i; the first rejection ends
+// the sweep.  The draw then re-reads row n (an L2 hit: one row is ~0.6 MB) together with
+// the draft row, forming p on the fly, with the same segment-sum / prefix / finish-inside
+// scheme as spec_accept_kernel.  Greedy mode (temperature 0) replaces max/sum by a
+// block-wide argmax (smallest index on ties) and needs neither q nor uniforms.
+// Exponentials are ex2.approx in fp32 with log2(e)/T folded into the argument; sums and
+// compares are fp64.  A decision can therefore differ from an all-fp64 evaluation only
+// within fp32 rounding of p at a decision or CDF boundary.
+#include <cuda_bf16.h>
+
+#include "nsd_internal.h"
+
+namespace nsd {
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+constexpr int kSeg = 128;                       // tokens per segment of the draw
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Four consecutive logits starting at token k0 (a multiple of 4); tokens past the vocabulary read as -inf.
+template <typename T>
+__device__ __forceinline__ float4 load4(const T* row, int k0, int vocab, bool vec_ok) {
+    float4 z;
+    if (vec_ok) {
+        if constexpr (sizeof(T) == 4) {
+            z = __ldg(reinterpret_cast<const float4*>(row + k0));
+        } else {
+            const uint2 raw = __ldg(reinterpret_cast<const uint2*>(row + k0));
+            const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+            const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+            z = make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
+        }
+    } else {
+        z.x = k0 + 0 < vocab ? to_float(row[k0 + 0]) : -INFINITY;
+        z.y = k0 + 1 < vocab ? to_float(row[k0 + 1]) : -INFINITY;
+        z.z = k0 + 2 < vocab ? to_float(row[k0 + 2]) : -INFINITY;
+        z.w = k0 + 3 < vocab ? to_float(row[k0 + 3]) : -INFINITY;
+    }
+    return z;
+}
+
+struct Shared {
+    float red_m[kWarps];
+    double red_s[kWarps];
+    int red_i[kWarps];
+    float row_max;        // M of the current row
+    double row_sum;       // S = sum_k 2^((z_k - M) * c)
+    int row_argmax;
+    int n;                // accepted length once decided, else -1
+    int found_seg;
+    int token;
+    double total;
+};
+
+// Block-wide max and sum of exponentials of one row: every thread keeps a running (m, s) pair.
+template <typename T>
+__device__ void row_stats(const T* row, int vocab, bool vec_ok, float c, Shared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float m = -INFINITY, s = 0.f;
+    const int n4 = (vocab + 3) / 4;
+#pragma unroll 4
+    for (int k4 = tid; k4 < n4; k4 += kThreads) {
+        const float4 z = load4(row, k4 * 4, vocab, vec_ok);
+        const float zm = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
+        if (zm > m) {
+            s *= ex2_approx((m - zm) * c);          // m = -inf: s is 0 and stays 0
+            m = zm;
+        }
+        if (m > -INFINITY)
+            s += ex2_approx((z.x - m) * c) + ex2_approx((z.y - m) * c) + ex2_approx((z.z - m) * c) + ex2_approx((z.w - m) * c);
+    }
+    float wm = m;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
+    double ws = (m > -INFINITY) ? (double)s * (double)ex2_approx((m - wm) * c) : 0.0;
+    ws = warp_sum(ws);
+    if (lane == 0) {
+        sh.red_m[warp] = wm;
+        sh.red_s[warp] = ws;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const float pm = lane < kWarps ? sh.red_m[lane] : -INFINITY;
+        float bm = pm;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
+        double bs = (lane < kWarps && pm > -INFINITY) ? sh.red_s[lane] * (double)ex2_approx((pm - bm) * c) : 0.0;
+        bs = warp_sum(bs);
+        if (lane == 0) {
+            sh.row_max = bm;
+            sh.row_sum = bs;
+        }
+    }
+    __syncthreads();
+}
+
+// Block-wide argmax of one row: largest value, smallest index among equals, NaN never wins.
+template <typename T>
+__device__ void row_argmax(const T* row, int vocab, bool vec_ok, Shared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float bv = -INFINITY;
+    int bi = -1;
+    const int n4 = (vocab + 3) / 4;
+    for (int k4 = tid; k4 < n4; k4 += kThreads) {
+        const float4 z = load4(row, k4 * 4, vocab, vec_ok);
+        const float v[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int k = k4 * 4 + j;
+            if (k < vocab && (v[j] > bv || (bi < 0 && v[j] == v[j]))) {      // strictly greater, or the first non-NaN
+                bv = v[j];
+                bi = k;
+            }
+        }
+    }
+    auto better = [](float v1, int i1, float v2, int i2) {   // is (v1, i1) ahead of (v2, i2)?
+        if (i1 < 0) return false;
+        if (i2 < 0) return true;
+        return v1 > v2 || (v1 == v2 && i1 < i2);
+    };
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (better(ov, oi, bv, bi)) bv = ov, bi = oi;
+    }
+    if (lane == 0) {
+        sh.red_m[warp] = bv;
+        sh.red_i[warp] = bi;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        bv = lane < kWarps ? sh.red_m[lane] : -INFINITY;
+        bi = lane < kWarps ? sh.red_i[lane] : -1;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (better(ov, oi, bv, bi)) bv = ov, bi = oi;
+        }
+        if (lane == 0) sh.row_argmax = bi;
+    }
+    __syncthreads();
+}
+
+}  // namespace
+}  // namespace nsd
+
+#include "spec_accept_logits_kernel.inc"
