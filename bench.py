@@ -158,13 +158,14 @@ def oracle_sample(cfg, meta, host, target_seconds):
     # spend about target_seconds: first more requests of layer 0, then further layers' query rows
     want = n_probe * max(target_seconds, t_probe) / max(t_probe, 1e-3)           # request-layers affordable
     n_attn = int(min(B, max(n_probe, want)))
-    n_layers = int(min(L, max(1, want // max(n_attn, 1))))
     sel = np.ascontiguousarray(order[:n_attn])
     keys_all = float((meta.ctx_len.astype(np.int64) + cfg.gamma + 1).sum())
     keys_sel = float((meta.ctx_len[sel].astype(np.int64) + cfg.gamma + 1).sum())
+    n_layers = 0
     t0 = time.perf_counter()
-    for l in range(n_layers):
-        oracle.verify_attn(pool, host["q"][l], meta.ctx_len, meta.kv_indptr, meta.kv_indices, cfg.gamma, layer=0, req_list=sel)
+    while n_layers < L and (n_layers == 0 or time.perf_counter() - t0 < target_seconds):
+        oracle.verify_attn(pool, host["q"][n_layers], meta.ctx_len, meta.kv_indptr, meta.kv_indices, cfg.gamma, layer=0, req_list=sel)
+        n_layers += 1
     t_attn = time.perf_counter() - t0
     t_attn_layer = t_attn / n_layers * keys_all / keys_sel   # attention cost is proportional to visible keys
     t0 = time.perf_counter()
