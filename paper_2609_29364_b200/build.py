@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnsd.so")
-SOURCES = ["nsd_api.cu", "kv_prepare.cu", "verify_attn.cu", "spec_accept.cu", "spec_accept_logits.cu", "nsd_schedule.cpp"]
+SOURCES = ["nsd_api.cu", "kv_prepare.cu", "verify_attn.cu", "verify_attn_umma.cu", "spec_accept.cu", "spec_accept_logits.cu", "nsd_schedule.cpp"]
 
 
 def _stale() -> bool:

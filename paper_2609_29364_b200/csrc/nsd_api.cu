@@ -41,6 +41,11 @@ struct nsd_ctx {
     cudaStream_t copy;         // uploads of the acceptance inputs in nsd_verify_round_host
     cudaEvent_t ev_start, ev_side_done, ev_plan_free, ev_copy_go, ev_accept_in;
     std::vector<cudaEvent_t> ev_prep, ev_attn;
+    // tcgen05 attention: one tensor map per layer slab of the pool last seen, and the SM count for the persistent grid
+    std::vector<CUtensorMap> tmaps;
+    std::vector<const void*> tmap_slab;
+    int n_sms;
+    int attn_path;             // 0 = mma.sync kernel, 1 = tcgen05 kernel where it applies
     int64_t launches;
     char err[256];
 };
@@ -194,6 +199,14 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     }
     if ((e = attn_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(attention)");
     if ((e = gather_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(gather)");
+    if ((e = attn_umma_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(tcgen05 attention)");
+    ctx->tmaps.resize(cfg->num_slabs);
+    ctx->tmap_slab.assign(cfg->num_slabs, nullptr);
+    if ((e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device)) != cudaSuccess) return fail(e, "cudaDeviceGetAttribute");
+    {
+        const char* path = getenv("NSD_ATTN_PATH");          // "mma" or "tcgen05"; default below
+        ctx->attn_path = path ? (strcmp(path, "tcgen05") == 0) : 0;
+    }
     *out = ctx;
     return NSD_OK;
 }
@@ -416,6 +429,21 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
     else if (subset == 1) { a.items = ctx->d_items_split; a.n_items = ctx->n_res; }
     else { a.items = ctx->d_items_split + ctx->n_res; a.n_items = ctx->n_mig_items; }
     if (a.n_items == 0) return NSD_OK;
+    if (ctx->attn_path == 1 && !fuse && ctx->cfg.head_dim == 128) {
+        const int slab = layer % ctx->cfg.num_slabs;
+        if (ctx->tmap_slab[slab] != a.pool_slab) {
+            ctx->tmap_slab[slab] = make_kv_tensor_map(&ctx->tmaps[slab], a.pool_slab, ctx->shape) ? a.pool_slab : nullptr;
+        }
+        if (ctx->tmap_slab[slab] == a.pool_slab) {
+            a.tmap = ctx->tmaps[slab];
+            a.tmap_valid = 1;
+        }
+        if (attn_umma_supported(a)) {
+            NSD_CUDA(ctx, launch_attn_umma(a, st, ctx->n_sms));
+            ctx->launches++;
+            return NSD_OK;
+        }
+    }
     NSD_CUDA(ctx, launch_attn(a, st));
     ctx->launches++;
     return NSD_OK;

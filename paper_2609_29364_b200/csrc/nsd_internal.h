@@ -1,5 +1,6 @@
 // Internal declarations shared by the library's translation units (not part of the ABI).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -55,6 +56,8 @@ struct AttnLaunch {
     int32_t* status;
     int32_t m_rows;              // (Hq/Hkv) * (gamma+1)
     int32_t tune_stages;         // experiment knob: 0 = default pipeline depth
+    int32_t tmap_valid;          // tmap describes pool_slab (tcgen05 path only)
+    CUtensorMap tmap;
 };
 
 cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const int32_t* src, const int32_t* dst,
@@ -69,6 +72,10 @@ cudaError_t launch_commit(const Shape& s, uint16_t* slab, int32_t batch, int32_t
                           cudaStream_t stream);
 cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream);
 cudaError_t gather_init();        // opt in to the copy ring's dynamic shared memory, once per device
+cudaError_t attn_umma_init();     // same for the tcgen05 attention kernels
+bool attn_umma_supported(const AttnLaunch& a);
+cudaError_t launch_attn_umma(const AttnLaunch& a, cudaStream_t stream, int n_sms);
+bool make_kv_tensor_map(CUtensorMap* map, const void* slab, const Shape& s);
 cudaError_t attn_init();          // opt in to large dynamic shared memory, once per process
 cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
                           const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int32_t* ctx_len,

@@ -1,0 +1,205 @@
+// Verification attention on the 5th-generation tensor cores (tcgen05 + TMEM + TMA).
+//
+// Same operation and same split-KV bookkeeping as verify_attn.cu (Appendix G.2: anchor +
+// proposal rows of a request attend its paged KV; Section 3: block maps), different engine.
+// The legacy mma.sync path tops out near 250 TFLOP/s under the board power cap, which is what
+// bounds the kernel once gamma reaches 6-8 (28-36 stacked rows); tcgen05.mma has an order of
+// magnitude more headroom and costs one issuing thread.
+//
+// "Keys on lanes".  A tile is 128 keys.  Both contractions put the long dimension on the 128
+// TMEM lanes and the few query rows on the columns:
+//     S^T[128 keys x R rows] = K[128 x 128] Q^T     A = K tile (K-major, 128B swizzle), B = Q (K-major)
+//     O^T[128 dims x R rows] += V^T[128 x 128 keys] P^T   A = V tile (MN-major), B = P^T (MN-major)
+// so every one of the 128 softmax threads owns one key (one TMEM lane) of S^T and one output
+// dimension of O^T; R = rows padded to 32 / 48 / 64 is only the column count.  TMEM use is
+// 2R <= 128 columns.
+//
+// One persistent CTA per SM, three roles:
+//   warp 4, one lane   producer: walks its work units (item, kv head) and their tiles, and for each
+//                      tile issues 32 TMA box loads (16 keys x 64 dims, 128-byte swizzle) of K and V
+//                      into a 3-stage ring (64 KiB per stage); blocks past the chunk are loaded
+//                      out of bounds, which zero-fills them;
+//   warp 5, one lane   MMA issuer: S^T = K Q^T when a stage is full; O^T += V^T P^T when the
+//                      softmax threads have published P^T; tcgen05.commit signals the mbarriers;
+//   warps 0-3          softmax: read S^T from TMEM, mask, exponentiate against a lazily refreshed
+//                      running maximum (refreshed, with an O^T rescale in TMEM, only when a score
+//                      exceeds it by 2^8), write P^T (bf16) to shared memory in the UMMA layout;
+//                      at the end of a unit reduce the row sums, read O^T and write the output or
+//                      the split-KV partial (the last CTA of a (request, head) merges).
+// The producer runs up to three tiles ahead, also across unit boundaries, so the HBM stream never
+// drains while a unit's epilogue runs.  Every mbarrier wait is bounded; on expiry the CTA raises an
+// abort flag, records STATUS_TIMEOUT, frees its TMEM and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "nsd_internal.h"
+
+namespace nsd {
+namespace {
+
+constexpr int kTileKeys = 128;
+constexpr int kBlockSizeU = 16;                         // keys per pool block
+constexpr int kBlocksPerTile = 8;
+constexpr int kStages = 3;
+constexpr int kHalfBytes = kTileKeys * 128;              // [128 keys][64 dims] bf16 = 16 KiB
+constexpr int kStageBytes = 4 * kHalfBytes;              // K lo, K hi, V lo, V hi
+constexpr int kSoftmaxThreads = 128;
+constexpr int kThreads = 192;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kMaxSlack = 8.0f;
+constexpr uint32_t kSpinLimit = 1u << 24;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ---- mbarrier / fences -------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait; gives up when the CTA's abort flag is raised or the poll budget runs out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if ((i & 63) == 63 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ bool softmax_bar_or(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbarrier.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return out != 0;
+}
+
+// ---- TMA -----------------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+                 : "memory");
+}
+
+// ---- tcgen05 ---------------------------------------------------------------------------------------
+// Shared-memory matrix descriptor: start address, leading / stride byte offsets (16-byte units),
+// descriptor version 1, layout type (0 = no swizzle, 2 = 128-byte swizzle).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32) | ((uint64_t)1 << 46) | ((uint64_t)(layout & 7) << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, majorness bits, N >> 3, M >> 4.
+__device__ __forceinline__ uint32_t instr_desc(int M, int N, int a_mn_major, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 16 consecutive columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15]))
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory carve-up for R query-row columns.
+template <int R>
+struct Layout {
+    static constexpr int kQHalfBytes = R * 128;                      // [R rows][64 dims]
+    static constexpr int kQBytes = 2 * kQHalfBytes;
+    static constexpr int kPBytes = kTileKeys * R * 2;                // P^T, bf16
+    static constexpr int kPLbo = (R / 8) * 128;                      // next 8 keys
+    static constexpr int kOffQ = kStages * kStageBytes;
+    static constexpr int kOffP = kOffQ + kQBytes;
+    static constexpr int kOffRed = kOffP + kPBytes;                  // [4 warps][R] floats: cross-warp reductions
+    static constexpr int kBytes = kOffRed + 4 * R * 4 + 1024;        // + slack for the 1024-byte alignment of the base
+};
+
+}  // namespace
+}  // namespace nsd
+
+#include "verify_attn_umma_kernel.inc"
+
+namespace nsd {
+
+cudaError_t attn_umma_init() {
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(verify_attn_umma_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, Layout<32>::kBytes)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(verify_attn_umma_kernel<48>, cudaFuncAttributeMaxDynamicSharedMemorySize, Layout<48>::kBytes)) != cudaSuccess) return e;
+    return cudaFuncSetAttribute(verify_attn_umma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Layout<64>::kBytes);
+}
+
+// Tensor map over one layer slab seen as a 2-D bf16 tensor [rows][128 dims], rows = (block, K|V, kv head, slot);
+// box = 16 rows x 64 dims with the 128-byte swizzle the UMMA descriptors expect.  Returns false when the driver
+// entry point is unavailable or refuses the shape (the caller then stays on the mma.sync kernel).
+bool make_kv_tensor_map(CUtensorMap* map, const void* slab, const Shape& s) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            fn = nullptr;
+        return reinterpret_cast<EncodeFn>(fn);
+    }();
+    if (!encode || s.D != 128 || s.bs != 16) return false;
+    const cuuint64_t dims[2] = {128, (cuuint64_t)s.num_blocks * 2 * s.Hkv * 16};
+    const cuuint64_t strides[1] = {256};
+    const cuuint32_t box[2] = {64, 16};
+    const cuuint32_t estr[2] = {1, 1};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(slab), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace nsd
