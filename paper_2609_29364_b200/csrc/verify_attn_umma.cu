@@ -47,7 +47,7 @@ constexpr int kSoftmaxThreads = 128;
 constexpr int kThreads = 192;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kMaxSlack = 8.0f;
-constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr uint32_t kSpinLimit = 1u << 20;          // wait slices of ~2 us each
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -70,17 +70,19 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait; gives up when the CTA's abort flag is raised or the poll budget runs out.
+// Bounded wait.  try_wait parks the thread in hardware until the phase completes or a time slice (hinted at
+// ~2 us) runs out, so waiting threads do not flood shared memory with polls; the slices are counted, and the
+// wait gives up when the CTA's abort flag is raised or the budget (a few seconds) is spent.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         uint32_t done;
         asm volatile(
-            "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(2000u)
             : "memory");
         if (done) return true;
-        if ((i & 63) == 63 && *abort_flag) return false;
+        if (*abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
@@ -157,10 +159,11 @@ struct Layout {
     static constexpr int kQHalfBytes = R * 128;                      // [R rows][64 dims]
     static constexpr int kQBytes = 2 * kQHalfBytes;
     static constexpr int kPBytes = kTileKeys * R * 2;                // P^T, bf16
+    static constexpr int kPBuffers = R <= 32 ? 2 : 1;                // two when shared memory allows
     static constexpr int kPLbo = (R / 8) * 128;                      // next 8 keys
     static constexpr int kOffQ = kStages * kStageBytes;
     static constexpr int kOffP = kOffQ + kQBytes;
-    static constexpr int kOffRed = kOffP + kPBytes;                  // [4 warps][R] floats: cross-warp reductions
+    static constexpr int kOffRed = kOffP + kPBuffers * kPBytes;      // [4 warps][R] floats: cross-warp reductions
     static constexpr int kBytes = kOffRed + 4 * R * 4 + 1024;        // + slack for the 1024-byte alignment of the base
 };
 

@@ -1,0 +1,50 @@
+"""GPU parity of the tcgen05 / TMEM / TMA attention kernel (opt-in: NSD_ATTN_PATH=tcgen05 when the
+context is created), against the same oracle and tolerance as the default kernel."""
+import numpy as np
+import pytest
+
+import workload as W
+import test_gpu_verify_attn as base
+import test_gpu_round as rnd
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _tcgen05_path(monkeypatch):
+    monkeypatch.setenv("NSD_ATTN_PATH", "tcgen05")
+
+
+@pytest.mark.parametrize("gamma", [1, 4, 6, 8, 11, 15])
+def test_row_counts_32_48_64(gamma):
+    """R = 32, 48 and 64 query-row columns; lengths around block, tile (128 keys) and chunk edges."""
+    cfg = base._cfg(f"u{gamma}", batch=11, gamma=gamma, ctx=("fixed", [0, 1, 15, 16, 111, 127, 128, 129, 300, 517, 1100]), seed=160 + gamma)
+    _, _, o, lse, res = base._run(cfg, want_lse=True)
+    base._check(o, res, lse)
+
+
+@pytest.mark.parametrize("chunk_blocks", [2, 6, 10, 16, 0])
+def test_split_kv_with_chunks_that_are_not_whole_tiles(chunk_blocks):
+    """Chunks of 2..16 blocks against 8-block tiles: keys past a chunk are zero-filled boxes and must be masked."""
+    cfg = base._cfg("usplit", batch=8, gamma=4, ctx=("fixed", [5, 40, 100, 257, 380, 600, 1023, 1500]), seed=172)
+    _, _, o, lse, res = base._run(cfg, chunk_blocks=chunk_blocks, want_lse=True)
+    base._check(o, res, lse)
+
+
+def test_many_units_per_cta_and_layers():
+    """More (item, head) units than SMs, so the persistent CTAs walk several units each, over aliased slabs."""
+    cfg = base._cfg("umany", batch=48, gamma=4, ctx=("uniform", 1, 700), layers=3, seed=173)
+    _, _, o, _, res = base._run(cfg, slabs=2, chunk_blocks=8)
+    base._check(o, res)
+
+
+def test_fused_round_and_poisoned_tail_slots():
+    rnd._run_round(rnd.MULTI, 2)
+    rnd._run_round(rnd.ALLMIG, 3)
+
+
+def test_group_size_one_and_eight():
+    for hq, hkv in ((8, 8), (8, 1)):
+        cfg = base._cfg(f"ug{hq}_{hkv}", batch=5, gamma=4, ctx=("uniform", 1, 400), hq=hq, hkv=hkv, d=128, seed=174)
+        _, _, o, _, res = base._run(cfg)
+        base._check(o, res)
