@@ -255,6 +255,7 @@ class VerifyContext:
     @staticmethod
     def round_args(**kw) -> RoundArgs:
         a = RoundArgs()
+        a._keepalive = [v for v in kw.values() if hasattr(v, "data_ptr")]    # the struct holds raw addresses only
         for name, _ in RoundArgs._fields_:
             v = kw.pop(name, None)
             if name in ("n_mig_blocks", "batch", "gamma", "fuse_gather", "reserved"):
