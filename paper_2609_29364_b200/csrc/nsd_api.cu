@@ -680,6 +680,7 @@ nsd_status nsd_get_status(nsd_ctx* ctx, void* stream, int32_t* first_bad_request
     NSD_CUDA(ctx, cudaStreamSynchronize(st));
     if (first_bad_request) *first_bad_request = ctx->h_status[1] - 1;
     if (ctx->h_status[0] & STATUS_TIMEOUT) return NSD_ERR_TIMEOUT;
+    if (ctx->h_status[0] & STATUS_LAYOUT) return NSD_ERR_UNSUPPORTED;     // the tcgen05 kernel found its shared memory unaligned
     return ctx->h_status[0] ? NSD_ERR_DEVICE_FAULT : NSD_OK;
 }
 

@@ -22,7 +22,7 @@ struct __align__(16) AttnItem {
 };
 
 // Device status word: [0] = error bits, [1] = first offending request (+1; 0 = none).
-enum : int32_t { STATUS_BAD_BLOCK = 1, STATUS_BAD_TOKEN = 2, STATUS_TIMEOUT = 4 };
+enum : int32_t { STATUS_BAD_BLOCK = 1, STATUS_BAD_TOKEN = 2, STATUS_TIMEOUT = 4, STATUS_LAYOUT = 8 };
 
 struct Shape {
     int32_t num_slabs, num_blocks, Hq, Hkv, D, bs;

@@ -2,33 +2,38 @@
 //
 // Same operation and same split-KV bookkeeping as verify_attn.cu (Appendix G.2: anchor +
 // proposal rows of a request attend its paged KV; Section 3: block maps), different engine.
-// The legacy mma.sync path tops out near 250 TFLOP/s under the board power cap, which is what
-// bounds the kernel once gamma reaches 6-8 (28-36 stacked rows); tcgen05.mma has an order of
-// magnitude more headroom and costs one issuing thread.
 //
-// "Keys on lanes".  A tile is 128 keys.  Both contractions put the long dimension on the 128
+// "Keys on lanes".  A tile is 128 keys.  Every contraction puts the long dimension on the 128
 // TMEM lanes and the few query rows on the columns:
-//     S^T[128 keys x R rows] = K[128 x 128] Q^T     A = K tile (K-major, 128B swizzle), B = Q (K-major)
-//     O^T[128 dims x R rows] += V^T[128 x 128 keys] P^T   A = V tile (MN-major), B = P^T (MN-major)
-// so every one of the 128 softmax threads owns one key (one TMEM lane) of S^T and one output
-// dimension of O^T; R = rows padded to 32 / 48 / 64 is only the column count.  TMEM use is
-// 2R <= 128 columns.
+//     S^T[128 keys x R rows]  = K[128 x 128] Q^T            A = K tile (K-major, 128B swizzle), B = Q (K-major)
+//     O^T[128 dims x R rows] += V^T[128 x 128 keys] P^T     A = V tile (MN-major), B = P^T (MN-major)
+//     L[128 x R rows]        += 1[128 x 128 keys] P^T       A = a block of ones, B = P^T
+// so each of the 128 softmax threads owns one key (one TMEM lane) of S^T, each epilogue thread one
+// output dimension of O^T, and the row sums L come out of the tensor core replicated on every lane
+// (no cross-thread reduction anywhere on the common path).  R = rows padded to 32 / 48 / 64.
 //
-// One persistent CTA per SM, three roles:
-//   warp 4, one lane   producer: walks its work units (item, kv head) and their tiles, and for each
-//                      tile issues 32 TMA box loads (16 keys x 64 dims, 128-byte swizzle) of K and V
-//                      into a 3-stage ring (64 KiB per stage); blocks past the chunk are loaded
-//                      out of bounds, which zero-fills them;
-//   warp 5, one lane   MMA issuer: S^T = K Q^T when a stage is full; O^T += V^T P^T when the
-//                      softmax threads have published P^T; tcgen05.commit signals the mbarriers;
-//   warps 0-3          softmax: read S^T from TMEM, mask, exponentiate against a lazily refreshed
-//                      running maximum (refreshed, with an O^T rescale in TMEM, only when a score
-//                      exceeds it by 2^8), write P^T (bf16) to shared memory in the UMMA layout;
-//                      at the end of a unit reduce the row sums, read O^T and write the output or
-//                      the split-KV partial (the last CTA of a (request, head) merges).
-// The producer runs up to three tiles ahead, also across unit boundaries, so the HBM stream never
-// drains while a unit's epilogue runs.  Every mbarrier wait is bounded; on expiry the CTA raises an
-// abort flag, records STATUS_TIMEOUT, frees its TMEM and returns.
+// One persistent CTA per SM, 13 warps, every role walks the same static list of work units
+// (chunk item, kv head):
+//   warp 8 / warp 9   K producer / V producer: 16 lanes each issue one TMA box (16 keys x 64 dims,
+//                     128-byte swizzle) per tile into their own ring of 32 KiB stages.  Two issuing
+//                     warps because one warp's TMA issue rate tops out near 39 GB/s per SM; K stages
+//                     are released as soon as S^T is computed, so the K stream runs up to three tiles
+//                     ahead of V and P^T is usually ready when a V tile lands: almost the whole ring
+//                     is in flight.  Blocks past the chunk are loaded out of bounds (zero fill).
+//   warp 12           stages Q of the unit after next into one of two swizzled Q buffers.
+//   warp 10           issues S^T = K Q^T into one of three TMEM score buffers, as soon as K lands.
+//   warp 11           issues O^T += V^T P^T and L += 1 P^T once P^T is published and V has landed;
+//                     zeroes V rows of slots that hold no token first (0 x NaN must not reach O^T).
+//   warps 0-3         softmax: read S^T, mask, P^T = 2^(s - m) in bf16 into shared memory in the UMMA
+//                     layout.  m is a per-row reference point (the unit's first key), not the running
+//                     maximum: the result is exact for any reference as long as nothing overflows, so
+//                     m is only raised (with a rescale of O^T and L in TMEM) when a score exceeds it by
+//                     2^24 -- one CTA-group vote per tile, the refresh itself is rare.
+//   warps 4-7         epilogue: O^T / L out of one of two TMEM accumulator sets into the output or the
+//                     split-KV partial; the last CTA of a (request, head) merges.  Runs beside the next
+//                     unit's main loop.
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their
+// loops, STATUS_TIMEOUT is recorded, TMEM is freed and the kernel returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -40,13 +45,14 @@ namespace {
 constexpr int kTileKeys = 128;
 constexpr int kBlockSizeU = 16;                         // keys per pool block
 constexpr int kBlocksPerTile = 8;
-constexpr int kStages = 3;
 constexpr int kHalfBytes = kTileKeys * 128;              // [128 keys][64 dims] bf16 = 16 KiB
-constexpr int kStageBytes = 4 * kHalfBytes;              // K lo, K hi, V lo, V hi
-constexpr int kSoftmaxThreads = 128;
-constexpr int kThreads = 192;
+constexpr int kStageBytes = 2 * kHalfBytes;              // one K or one V tile: dims 0-63, dims 64-127
+constexpr int kSoftmaxThreads = 128;                     // warps 0-3
+constexpr int kEpilogueThreads = 128;                    // warps 4-7
+constexpr int kWarpK = 8, kWarpV = 9, kWarpS = 10, kWarpPV = 11, kWarpQ = 12;
+constexpr int kThreads = 13 * 32;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kMaxSlack = 8.0f;
+constexpr float kMaxSlack = 24.0f;                       // a score may exceed its row's reference by 2^24
 constexpr uint32_t kSpinLimit = 1u << 20;          // wait slices of ~2 us each
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -82,23 +88,62 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             : "r"(bar), "r"(parity), "r"(2000u)
             : "memory");
         if (done) return true;
+#ifdef NSD_UMMA_BACKOFF
+        __nanosleep(NSD_UMMA_BACKOFF);
+#endif
         if (*abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
 }
+#ifdef NSD_UMMA_PROF
+// Development aid: per-role wait and section times of CTA 0, kept in registers and flushed once at the end.
+__device__ long long g_prof[64];
+__device__ __forceinline__ bool mbar_wait_p(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long& acc, bool rec) {
+    const long long t0 = clock64();
+    const bool r = mbar_wait(bar, parity, abort_flag);
+    if (rec) acc += clock64() - t0;
+    return r;
+}
+#define PROF_DECL() long long prof_acc[32] = {0}
+#define PROF_FLUSH() do { if (blockIdx.x == 0) { _Pragma("unroll") for (int i_ = 0; i_ < 32; ++i_) if (prof_acc[i_]) atomicAdd(reinterpret_cast<unsigned long long*>(&g_prof[i_]), (unsigned long long)prof_acc[i_]); } } while (0)
+#define MBAR_WAIT(bar, par, ab, slot, rec) mbar_wait_p(bar, par, ab, prof_acc[slot], rec)
+#define PROF_NOW() clock64()
+#define PROF_ACC(slot, t0, rec) do { if (rec) prof_acc[slot] += clock64() - (t0); } while (0)
+#define PROF_INC(slot, rec) do { if (rec) prof_acc[slot] += 1; } while (0)
+#else
+#define PROF_DECL() do {} while (0)
+#define PROF_FLUSH() do {} while (0)
+#define MBAR_WAIT(bar, par, ab, slot, rec) mbar_wait(bar, par, ab)
+#define PROF_NOW() 0ll
+#define PROF_ACC(slot, t0, rec) do { (void)(t0); } while (0)
+#define PROF_INC(slot, rec) do {} while (0)
+#endif
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-__device__ __forceinline__ bool softmax_bar_or(bool pred) {
+// Named barriers of the two 128-thread groups: id 1 = softmax warps, id 2 = epilogue warps.
+template <int ID>
+__device__ __forceinline__ void group_bar_sync() { asm volatile("bar.sync %0, 128;" ::"n"(ID) : "memory"); }
+template <int ID>
+__device__ __forceinline__ bool group_bar_or(bool pred) {
     uint32_t out;
     asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbarrier.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbarrier.red.or.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(out)
-        : "r"((uint32_t)pred)
+        : "r"((uint32_t)pred), "n"(ID)
         : "memory");
     return out != 0;
+}
+
+// Bounded rendezvous of the four softmax warps on an mbarrier (one arrival per warp); false once the CTA is aborting.
+// The result is the same for every lane of a warp.
+__device__ __forceinline__ bool group_sync(uint32_t bar, uint32_t& phase, int lane, volatile int* abort_flag) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+    const bool ok = mbar_wait(bar, phase & 1, abort_flag);
+    ++phase;
+    return !__any_sync(0xffffffffu, !ok);
 }
 
 // ---- TMA -----------------------------------------------------------------------------------------
@@ -153,19 +198,31 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) 
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
-// Shared-memory carve-up for R query-row columns.
+// Shared-memory and TMEM carve-up for R query-row columns.
 template <int R>
 struct Layout {
+    static constexpr int kKStages = R <= 32 ? 3 : 2;
+    static constexpr int kVStages = 3;
     static constexpr int kQHalfBytes = R * 128;                      // [R rows][64 dims]
     static constexpr int kQBytes = 2 * kQHalfBytes;
     static constexpr int kPBytes = kTileKeys * R * 2;                // P^T, bf16
-    static constexpr int kPBuffers = R <= 32 ? 2 : 1;                // two when shared memory allows
     static constexpr int kPLbo = (R / 8) * 128;                      // next 8 keys
-    static constexpr int kOffQ = kStages * kStageBytes;
-    static constexpr int kOffP = kOffQ + kQBytes;
-    static constexpr int kOffRed = kOffP + kPBuffers * kPBytes;      // [4 warps][R] floats: cross-warp reductions
-    static constexpr int kBytes = kOffRed + 4 * R * 4 + 1024;        // + slack for the 1024-byte alignment of the base
+    static constexpr int kOffK = 0;
+    static constexpr int kOffV = kOffK + kKStages * kStageBytes;
+    static constexpr int kOffQ = kOffV + kVStages * kStageBytes;     // two buffers
+    static constexpr int kOffP = kOffQ + 2 * kQBytes;                // two buffers
+    static constexpr int kOffRed = kOffP + 2 * kPBytes;              // [4 warps][R] floats: tile maxima of a refresh
+    static constexpr int kOffRedE = kOffRed + 4 * R * 4;             // [4 warps][R] floats: the epilogue's row-sum reduction
+    static constexpr int kOffMref = kOffRedE + 4 * R * 4;            // [2][R] floats: minus the rows' reference points
+    static constexpr int kOffBars = kOffMref + 2 * R * 4;            // 40 mbarrier slots, then five words
+    static constexpr int kBytes = kOffBars + 40 * 8 + 32;
+    // TMEM columns: three S^T buffers, two O^T accumulators, two sets of per-key row-sum shares.
+    static constexpr int kTmemStride = R <= 32 ? 32 : 64;
+    static constexpr int kTmemCols = R <= 32 ? 256 : 512;
+    static constexpr int kTmemS = 0, kTmemO = 3 * kTmemStride, kTmemL = 5 * kTmemStride;
 };
+static_assert(Layout<32>::kBytes <= 227 * 1024 && Layout<48>::kBytes <= 227 * 1024 && Layout<64>::kBytes <= 227 * 1024,
+              "shared memory budget");
 
 }  // namespace
 }  // namespace nsd
@@ -206,3 +263,14 @@ bool make_kv_tensor_map(CUtensorMap* map, const void* slab, const Shape& s) {
 }
 
 }  // namespace nsd
+
+#ifdef NSD_UMMA_PROF
+extern "C" void nsd_debug_umma_prof(long long* out, int reset) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, nsd::g_prof, sizeof(long long) * 64);
+    if (reset) {
+        long long z[64] = {0};
+        cudaMemcpyToSymbol(nsd::g_prof, z, sizeof(z));
+    }
+}
+#endif
