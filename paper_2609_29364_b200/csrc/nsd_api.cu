@@ -38,9 +38,10 @@ struct nsd_ctx {
     int64_t plan_src_blocks;   // source blocks of the planned batch's reassigned requests
     // streams / events
     cudaStream_t side;
-    cudaStream_t copy;         // uploads of the acceptance inputs in nsd_verify_round_host
-    cudaEvent_t ev_start, ev_side_done, ev_plan_free, ev_copy_go, ev_accept_in;
+    cudaStream_t copy, down;   // nsd_verify_round_host: uploads in the order they are needed / per-layer read-back of o
+    cudaEvent_t ev_start, ev_side_done, ev_plan_free, ev_copy_go, ev_accept_in, ev_tables, ev_down_done;
     std::vector<cudaEvent_t> ev_prep, ev_attn;
+    std::vector<cudaEvent_t> ev_in, ev_out;    // nsd_verify_round_host: layer l's inputs have landed / its output is complete
     // tcgen05 attention: one tensor map per layer slab of the pool last seen, and the SM count for the persistent grid
     std::vector<CUtensorMap> tmaps;
     std::vector<const void*> tmap_slab;
@@ -169,7 +170,8 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     ctx->h_status = nullptr;
     ctx->side = nullptr;
     ctx->copy = nullptr;
-    ctx->ev_start = ctx->ev_side_done = ctx->ev_plan_free = ctx->ev_copy_go = ctx->ev_accept_in = nullptr;
+    ctx->ev_start = ctx->ev_side_done = ctx->ev_plan_free = ctx->ev_copy_go = ctx->ev_accept_in = ctx->ev_tables = ctx->ev_down_done = nullptr;
+    ctx->down = nullptr;
 
     auto fail = [&](cudaError_t e, const char* what) {
         nsd_status s = cuda_fail(ctx, e, what);
@@ -186,6 +188,9 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     if ((e = cudaMallocHost(&ctx->h_status, 4 * sizeof(int32_t))) != cudaSuccess) return fail(e, "cudaMallocHost(status)");
     if ((e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking)) != cudaSuccess) return fail(e, "cudaStreamCreate");
     if ((e = cudaStreamCreateWithFlags(&ctx->copy, cudaStreamNonBlocking)) != cudaSuccess) return fail(e, "cudaStreamCreate");
+    if ((e = cudaStreamCreateWithFlags(&ctx->down, cudaStreamNonBlocking)) != cudaSuccess) return fail(e, "cudaStreamCreate");
+    if ((e = cudaEventCreateWithFlags(&ctx->ev_tables, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+    if ((e = cudaEventCreateWithFlags(&ctx->ev_down_done, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     if ((e = cudaEventCreateWithFlags(&ctx->ev_copy_go, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     if ((e = cudaEventCreateWithFlags(&ctx->ev_accept_in, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     if ((e = cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
@@ -193,9 +198,13 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     if ((e = cudaEventCreateWithFlags(&ctx->ev_plan_free, cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     ctx->ev_prep.assign(cfg->num_layers, nullptr);
     ctx->ev_attn.assign(cfg->num_layers, nullptr);
+    ctx->ev_in.assign(cfg->num_layers, nullptr);
+    ctx->ev_out.assign(cfg->num_layers, nullptr);
     for (int l = 0; l < cfg->num_layers; ++l) {
         if ((e = cudaEventCreateWithFlags(&ctx->ev_prep[l], cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
         if ((e = cudaEventCreateWithFlags(&ctx->ev_attn[l], cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+        if ((e = cudaEventCreateWithFlags(&ctx->ev_in[l], cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
+        if ((e = cudaEventCreateWithFlags(&ctx->ev_out[l], cudaEventDisableTiming)) != cudaSuccess) return fail(e, "cudaEventCreate");
     }
     if ((e = attn_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(attention)");
     if ((e = gather_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(gather)");
@@ -215,6 +224,11 @@ nsd_status nsd_destroy(nsd_ctx* ctx) {
     if (!ctx) return NSD_OK;
     if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
     if (ctx->copy) { cudaStreamSynchronize(ctx->copy); cudaStreamDestroy(ctx->copy); }
+    if (ctx->down) { cudaStreamSynchronize(ctx->down); cudaStreamDestroy(ctx->down); }
+    if (ctx->ev_tables) cudaEventDestroy(ctx->ev_tables);
+    if (ctx->ev_down_done) cudaEventDestroy(ctx->ev_down_done);
+    for (auto ev : ctx->ev_in) if (ev) cudaEventDestroy(ev);
+    for (auto ev : ctx->ev_out) if (ev) cudaEventDestroy(ev);
     if (ctx->ev_copy_go) cudaEventDestroy(ctx->ev_copy_go);
     if (ctx->ev_accept_in) cudaEventDestroy(ctx->ev_accept_in);
     for (auto ev : ctx->ev_prep) if (ev) cudaEventDestroy(ev);
@@ -500,11 +514,13 @@ nsd_status nsd_spec_accept_logits(nsd_ctx* ctx, const void* logits, int32_t logi
 }
 
 namespace {
-// What the host-buffer variant slips in between the last layer and the acceptance.
+// What the host-buffer variant threads through the round: every layer waits for its own inputs (uploaded on the
+// copy stream in the order of use), its output is read back on a third stream as soon as it is complete, and the
+// acceptance waits for its inputs, which follow the layers' on the copy stream.
 struct BeforeAccept {
-    void* h_o;                 // read the attention output back as soon as the layers are done
-    size_t o_bytes;
-    cudaEvent_t inputs_ready;  // the acceptance inputs arrive on another stream
+    void* h_o;                 // host destination of the attention output
+    size_t o_layer_bytes;
+    cudaEvent_t inputs_ready;  // the acceptance inputs have landed
 };
 nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const BeforeAccept* hook);
 }  // namespace
@@ -546,6 +562,10 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
     }
     for (int l = 0; l < L; ++l) {
         uint16_t* slab = slab_ptr(ctx, a->kv_pool, l);
+        if (hook) {
+            NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_in[l], 0));
+            if (overlap) NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_in[l], 0));
+        }
         if (overlap) {
             // side stream: copy + append of the reassigned requests of layer l
             if (l >= S) NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_attn[l - S], 0));
@@ -584,14 +604,21 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
                                         a->kv_indptr, a->kv_indices, l, 0, st);
             if (s != NSD_OK) return s;
         }
+        if (hook) {
+            NSD_CUDA(ctx, cudaEventRecord(ctx->ev_out[l], st));
+            NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->down, ctx->ev_out[l], 0));
+            NSD_CUDA(ctx, cudaMemcpyAsync(static_cast<char*>(hook->h_o) + (size_t)l * hook->o_layer_bytes, o + l * q_layer,
+                                          hook->o_layer_bytes, cudaMemcpyDeviceToHost, ctx->down));
+        }
     }
     if (hook) {
-        NSD_CUDA(ctx, cudaMemcpyAsync(hook->h_o, a->o, hook->o_bytes, cudaMemcpyDeviceToHost, st));
+        NSD_CUDA(ctx, cudaEventRecord(ctx->ev_down_done, ctx->down));
         NSD_CUDA(ctx, cudaStreamWaitEvent(st, hook->inputs_ready, 0));
     }
     NSD_CUDA(ctx, launch_accept(a->p, a->q_draft, a->draft_tok, a->u_acc, a->u_smp, batch, gamma, ctx->cfg.vocab_size,
                                 a->ctx_len, a->acc_len, a->out_tok, a->new_ctx_len, ctx->d_status, st));
     ctx->launches++;
+    if (hook) NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down_done, 0));      // the caller's stream covers the read-back
     return NSD_OK;
 }
 }  // namespace
@@ -610,49 +637,60 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
     const int64_t V = ctx->cfg.vocab_size, rows = (int64_t)batch * (gamma + 1);
     int64_t up = 0, down = 0;
     struct Copy { const void* src; const void* dst; int64_t bytes; };
-    // The first nine feed the layers and go ahead of them on `stream`; the last five feed only the acceptance and
-    // travel on the copy stream while the layers run.
-    constexpr int kLayerInputs = 9;
-    const Copy ups[] = {
+    // Everything goes up on the copy stream in the order it is needed: the tables, then layer by layer the new K / V
+    // rows and the queries (each layer starts as soon as its own inputs have landed), then the acceptance inputs,
+    // which travel while the layers run.  The output comes back layer by layer on a third stream.
+    const int64_t kv_layer_bytes = rows * Hkv * D * 2, q_layer_bytes = rows * Hq * D * 2;
+    const Copy tables[] = {
         {h->ctx_len, d->ctx_len, batch * 4LL},
         {h->kv_indptr, d->kv_indptr, (batch + 1) * 8LL},
         {h->kv_indices, d->kv_indices, total_table_entries * 4},
         {h->is_migrated, d->is_migrated, h->is_migrated ? batch * 1LL : 0},
         {h->mig_src, d->mig_src, h->n_mig_blocks * 4},
         {h->mig_dst, d->mig_dst, h->n_mig_blocks * 4},
-        {h->k_new, d->k_new, L * rows * Hkv * D * 2},
-        {h->v_new, d->v_new, L * rows * Hkv * D * 2},
-        {h->q, d->q, L * rows * Hq * D * 2},
+    };
+    const Copy accept_in[] = {
         {h->p, d->p, (int64_t)batch * (gamma + 1) * V * 4},
         {h->q_draft, d->q_draft, (int64_t)batch * gamma * V * 4},
         {h->draft_tok, d->draft_tok, (int64_t)batch * gamma * 4},
         {h->u_acc, d->u_acc, (int64_t)batch * gamma * 4},
         {h->u_smp, d->u_smp, batch * 4LL},
     };
-    for (const Copy& c : ups) {
-        if (c.bytes == 0) continue;
-        if (!c.src || !c.dst) return NSD_ERR_INVALID_ARG;
-    }
+    for (const Copy& c : tables)
+        if (c.bytes != 0 && (!c.src || !c.dst)) return NSD_ERR_INVALID_ARG;
+    for (const Copy& c : accept_in)
+        if (c.bytes != 0 && (!c.src || !c.dst)) return NSD_ERR_INVALID_ARG;
+    if (!h->k_new || !d->k_new || !h->v_new || !d->v_new || !h->q || !d->q) return NSD_ERR_INVALID_ARG;
     if (!h->o || !d->o || !h->acc_len || !d->acc_len || !h->out_tok || !d->out_tok) return NSD_ERR_INVALID_ARG;
     nsd_status s = nsd_verify_plan(ctx, batch, gamma, h->ctx_len, h->kv_indptr, h->is_migrated, 0, stream);
     if (s != NSD_OK) return s;
     NSD_CUDA(ctx, cudaEventRecord(ctx->ev_copy_go, st));          // the device buffers are free once prior work is done
     NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->copy, ctx->ev_copy_go, 0));
-    int idx = 0;
-    for (const Copy& c : ups) {
-        cudaStream_t target = idx++ < kLayerInputs ? st : ctx->copy;
-        if (c.bytes == 0) continue;
-        NSD_CUDA(ctx, cudaMemcpyAsync(const_cast<void*>(c.dst), c.src, (size_t)c.bytes, cudaMemcpyHostToDevice, target));
+    NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->down, ctx->ev_copy_go, 0));
+    auto upload = [&](const Copy& c) -> cudaError_t {
+        if (c.bytes == 0) return cudaSuccess;
         up += c.bytes;
+        return cudaMemcpyAsync(const_cast<void*>(c.dst), c.src, (size_t)c.bytes, cudaMemcpyHostToDevice, ctx->copy);
+    };
+    for (const Copy& c : tables) NSD_CUDA(ctx, upload(c));
+    NSD_CUDA(ctx, cudaEventRecord(ctx->ev_tables, ctx->copy));
+    NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_tables, 0));
+    for (int l = 0; l < L; ++l) {
+        NSD_CUDA(ctx, upload({static_cast<const char*>(h->k_new) + l * kv_layer_bytes, static_cast<const char*>(d->k_new) + l * kv_layer_bytes, kv_layer_bytes}));
+        NSD_CUDA(ctx, upload({static_cast<const char*>(h->v_new) + l * kv_layer_bytes, static_cast<const char*>(d->v_new) + l * kv_layer_bytes, kv_layer_bytes}));
+        NSD_CUDA(ctx, upload({static_cast<const char*>(h->q) + l * q_layer_bytes, static_cast<const char*>(d->q) + l * q_layer_bytes, q_layer_bytes}));
+        NSD_CUDA(ctx, cudaEventRecord(ctx->ev_in[l], ctx->copy));
     }
+    for (const Copy& c : accept_in) NSD_CUDA(ctx, upload(c));
     NSD_CUDA(ctx, cudaEventRecord(ctx->ev_accept_in, ctx->copy));
-    const BeforeAccept hook{h->o, (size_t)(L * rows * Hq * D * 2), ctx->ev_accept_in};
+    const BeforeAccept hook{h->o, (size_t)q_layer_bytes, ctx->ev_accept_in};
     s = round_impl(ctx, d, stream, &hook);
     if (s != NSD_OK) {
         cudaStreamSynchronize(ctx->copy);
+        cudaStreamSynchronize(ctx->down);
         return s;
     }
-    down += (int64_t)hook.o_bytes;
+    down += (int64_t)hook.o_layer_bytes * L;
     const Copy downs[] = {
         {d->acc_len, h->acc_len, batch * 4LL},
         {d->out_tok, h->out_tok, rows * 4},
