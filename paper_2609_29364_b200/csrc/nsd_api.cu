@@ -263,6 +263,7 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
         total_blocks += need;
     }
     if (batch > 0 && h_kv_indptr[batch] > ctx->cfg.max_table_entries) return NSD_ERR_CAPACITY;
+    if (batch > 0 && h_kv_indptr[batch] > INT32_MAX) return NSD_ERR_CAPACITY;      // items carry table offsets as int32
 
     // ---- chunk length: enough items to fill the machine several times over, long enough
     //      that the fp32 partials of split requests stay a small fraction of the KV bytes
@@ -309,6 +310,8 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
             it.chunk_idx = c;
             it.nchunks = n_eff;
             it.src_off = (int32_t)src_off;
+            it.ctx = h_ctx_len[r];
+            it.tbl_off = (int32_t)h_kv_indptr[r];
             items.push_back({it, h_is_migrated ? (h_is_migrated[r] != 0) : 0});
         }
         if (n_eff > 1) slot += n_eff;
