@@ -3,14 +3,13 @@
 // Same operation and same split-KV bookkeeping as verify_attn.cu (Appendix G.2: anchor +
 // proposal rows of a request attend its paged KV; Section 3: block maps), different engine.
 //
-// "Keys on lanes".  A tile is 128 keys.  Every contraction puts the long dimension on the 128
+// "Keys on lanes".  A tile is 128 keys.  Both contractions put the long dimension on the 128
 // TMEM lanes and the few query rows on the columns:
 //     S^T[128 keys x R rows]  = K[128 x 128] Q^T            A = K tile (K-major, 128B swizzle), B = Q (K-major)
 //     O^T[128 dims x R rows] += V^T[128 x 128 keys] P^T     A = V tile (MN-major), B = P^T (MN-major)
-//     L[128 x R rows]        += 1[128 x 128 keys] P^T       A = a block of ones, B = P^T
-// so each of the 128 softmax threads owns one key (one TMEM lane) of S^T, each epilogue thread one
-// output dimension of O^T, and the row sums L come out of the tensor core replicated on every lane
-// (no cross-thread reduction anywhere on the common path).  R = rows padded to 32 / 48 / 64.
+// so each of the 128 softmax threads owns one key (one TMEM lane) of S^T and each epilogue thread
+// one output dimension of O^T.  R = rows padded to 32 / 48 / 64.  tcgen05.mma costs its issuing
+// thread ~80 cycles whatever N is, so the instruction count per tile (8 + 8) is what matters.
 //
 // One persistent CTA per SM, 13 warps, every role walks the same static list of work units
 // (chunk item, kv head):
@@ -20,20 +19,24 @@
 //                     are released as soon as S^T is computed, so the K stream runs up to three tiles
 //                     ahead of V and P^T is usually ready when a V tile lands: almost the whole ring
 //                     is in flight.  Blocks past the chunk are loaded out of bounds (zero fill).
-//   warp 12           stages Q of the unit after next into one of two swizzled Q buffers.
+//   warp 12           stages Q of the next unit into one of two swizzled Q buffers.
 //   warp 10           issues S^T = K Q^T into one of three TMEM score buffers, as soon as K lands.
-//   warp 11           issues O^T += V^T P^T and L += 1 P^T once P^T is published and V has landed;
-//                     zeroes V rows of slots that hold no token first (0 x NaN must not reach O^T).
+//   warp 11           issues O^T += V^T P^T once P^T is published and V has landed; zeroes V rows of
+//                     slots that hold no token first (0 x NaN must not reach O^T).
 //   warps 0-3         softmax: read S^T, mask, P^T = 2^(s - m) in bf16 into shared memory in the UMMA
-//                     layout.  m is a per-row reference point (the unit's first key), not the running
-//                     maximum: the result is exact for any reference as long as nothing overflows, so
-//                     m is only raised (with a rescale of O^T and L in TMEM) when a score exceeds it by
-//                     2^24 -- one CTA-group vote per tile, the refresh itself is rare.
-//   warps 4-7         epilogue: O^T / L out of one of two TMEM accumulator sets into the output or the
-//                     split-KV partial; the last CTA of a (request, head) merges.  Runs beside the next
-//                     unit's main loop.
+//                     layout.  m is a per-row reference point (the score of the unit's first key), not
+//                     the running maximum: the result is exact for any reference as long as nothing
+//                     overflows, so the common tile needs no cross-thread reduction.  The four warps
+//                     vote through a split-phase mbarrier on whether a score outgrew its reference by
+//                     2^24 while the weights are already being formed; only then (rare) the references
+//                     are raised, O^T is rescaled in TMEM and the tile is redone.  Row sums are kept per
+//                     thread and left on the thread's TMEM lane at the end of the unit.
+//   warps 4-7         epilogue: add the 128 lanes' row-sum shares up, O^T / sum out of one of two TMEM
+//                     accumulator sets into the output or the split-KV partial; the last CTA of a
+//                     (request, head) merges.  Runs beside the next unit's main loop.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their
-// loops, STATUS_TIMEOUT is recorded, TMEM is freed and the kernel returns.
+// loops, STATUS_TIMEOUT is recorded, TMEM is freed and the kernel returns.  The softmax warps
+// rendezvous on mbarriers (bounded), never on named barriers, so an aborting CTA cannot hang.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
