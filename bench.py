@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--slabs", type=int, default=0, help="physical layer slabs (0 = as many as fit in 80%% of free memory)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-scheduled", action="store_true", help="skip the scheduler-driven two-bank rounds leg")
+    ap.add_argument("--scheduled-rounds", type=int, default=8)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target CPU time of the oracle sample")
     ap.add_argument("--batch", type=int, default=0, help="profiling only: override the batch size (not a bench line)")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: override the layer count (not a bench line)")
@@ -240,6 +242,72 @@ def workload_config(cfg, meta, slabs):
 
 
 # ----------------------------------------------------------------------------- our arm
+
+def scheduled_rounds_leg(cfg, device, rounds, d_accept):
+    """Rounds chosen by Algorithm 1 on a two-bank worker (paper_2609_29364_b200/rounds.py): the copy of batch k+1 into
+    the standby bank overlaps the run of batch k, the accepted suffix of batch k-1 is exported beside both.  Reports
+    the run time and the exposed KV-ready wait (Appendix G.2) per round.  Timing only: parity of this path is
+    tests/test_gpu_scheduled_rounds.py."""
+    import torch
+
+    import paper_2609_29364_b200 as nsd
+    from paper_2609_29364_b200.rounds import ScheduledRounds
+    from workload.banks import BankedPool
+
+    B, g, L = max(4, cfg.batch // 2), cfg.gamma, cfg.num_layers
+    n_req = (5 * B) // 2                                     # 2.5 batches in the stage's pool: about half of a batch comes back resident
+    ctx0 = W.draw_ctx_len(W.RoundConfig(**{**cfg.__dict__, "batch": n_req, "seed": cfg.seed + 7}))
+    max_new = rounds * (g + 1)
+    need = np.sort((ctx0.astype(np.int64) + max_new + g + 1 + cfg.block_size - 1) // cfg.block_size)[::-1]
+    bank_blocks = int(need[:B].sum()) + 64
+    banks = BankedPool(ctx0, g, cfg.block_size, max_new, bank_blocks, seed=cfg.seed)
+    slab_bytes = banks.num_blocks * cfg.block_elems * 2
+    free, _ = torch.cuda.mem_get_info(device)
+    slabs = int(min(L, 4, max(1, (0.6 * free) // slab_bytes)))
+    if L > 1 and slabs < 2:
+        return {"skipped": "not enough free device memory for two layer slabs"}
+    ctx = nsd.VerifyContext(num_layers=L, num_slabs=slabs, num_q_heads=cfg.num_q_heads, num_kv_heads=cfg.num_kv_heads,
+                            head_dim=cfg.head_dim, block_size=cfg.block_size, num_blocks=banks.num_blocks,
+                            region_b_begin=banks.region_b_begin, max_batch=B, max_gamma=g, vocab_size=cfg.vocab,
+                            max_table_entries=bank_blocks, device=str(device))
+    pool = torch.empty((slabs, banks.num_blocks * cfg.block_elems), dtype=torch.bfloat16, device=device)
+    for s_ in range(slabs):
+        pool[s_].normal_()
+    pool = pool.view(torch.int16)
+    rows = B * (g + 1)
+    rnd = lambda *shape: torch.randn(shape, dtype=torch.bfloat16, device=device).view(torch.int16)
+    fixed = dict(k_new=rnd(L, rows, cfg.num_kv_heads, cfg.head_dim), v_new=rnd(L, rows, cfg.num_kv_heads, cfg.head_dim),
+                 q=rnd(L, rows, cfg.num_q_heads, cfg.head_dim), p=d_accept["p"][:B], q_draft=d_accept["q_draft"][:B],
+                 draft_tok=d_accept["draft_tok"][:B], u_acc=d_accept["u_acc"][:B], u_smp=d_accept["u_smp"][:B])
+
+    def inputs(k, batch):
+        n = len(batch)
+        if n == B:
+            return fixed
+        cut = {name: fixed[name][:, :n * (g + 1)].contiguous() for name in ("k_new", "v_new", "q")}
+        cut.update({name: fixed[name][:n] for name in ("p", "q_draft", "draft_tok", "u_acc", "u_smp")})
+        return cut
+
+    recs = ScheduledRounds(ctx, pool, banks, ctx0, g, B, inputs, keep_outputs=False).run(rounds)
+    steady = recs[2:] if len(recs) > 3 else recs
+    blk_bytes = cfg.block_elems * 2 * L
+    out = {
+        "what": "Algorithm 1 picks each batch from a pool of %d requests; batch k runs out of bank k %% 2 while batch k+1's "
+                "non-resident requests are copied from the store into the other bank and batch k-1's accepted suffix is exported" % n_req,
+        "rounds": len(recs), "max_batch": B, "layers": L, "physical_layer_slabs": slabs,
+        "batch_sizes": [len(r.batch) for r in recs],
+        "resident_fraction": [round(float(r.entry.resident.mean()), 3) for r in recs],
+        "copied_GB": [round(r.copied_blocks * blk_bytes / 1e9, 2) for r in recs],
+        "run_ms": [round(r.run_ms, 3) for r in recs],
+        "exposed_kv_wait_ms": [round(r.exposed_wait_ms, 3) for r in recs],
+        "steady_state": {"run_ms_median": float(np.median([r.run_ms for r in steady])),
+                         "exposed_kv_wait_ms_median": float(np.median([r.exposed_wait_ms for r in steady])),
+                         "req_per_s": float(np.mean([len(r.batch) for r in steady]) / (np.median([r.run_ms for r in steady]) * 1e-3))},
+    }
+    ctx.close()
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -443,6 +511,25 @@ def run_ours(args):
                "h2d_bytes_per_step": int(moved["up"]), "d2h_bytes_per_step": int(moved["down"]),
                "api": "nsd_verify_round_host (pinned host buffers; the KV pool is worker state and stays in HBM)"}
 
+    # ---- rounds driven by the scheduler on a two-bank worker (rank 0, N = 1 only; needs the big pool's memory)
+    scheduled = None
+    if rank == 0 and world == 1 and not args.no_scheduled:
+        d_accept = {k_: d[k_] for k_ in ("p", "q_draft", "draft_tok", "u_acc", "u_smp")}
+        barrier()
+        ctx.close()
+        del pool, d_args, nomig, fused_args                   # everything that pins the big pool
+        try:
+            del graph
+        except NameError:
+            pass
+        try:
+            del h_args, h
+        except NameError:
+            pass
+        d.clear()
+        torch.cuda.empty_cache()
+        scheduled = scheduled_rounds_leg(cfg, device, args.scheduled_rounds, d_accept)
+
     # ---- the oracle on the host cores (rank 0, N = 1 only)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -486,6 +573,7 @@ def run_ours(args):
                 "speedup_over_headline": ms_round / ms_round_fused},
             "round_cuda_graph": None if ms_round_graph is None else {
                 "ms_per_step": ms_round_graph, "value": n_gpus * B / (ms_round_graph * 1e-3), "unit": "req/s"},
+            "scheduled_rounds": scheduled,
             "e2e": e2e, "gpu_launches": int(gpu_launches), "clocks": clocks, "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))

@@ -12,6 +12,7 @@ from .gen import (  # noqa: F401
     RoundConfig,
     accept_inputs,
     bf16_to_f32,
+    draw_ctx_len,
     export_tables,
     f32_to_bf16,
     make_batch_meta,

@@ -165,6 +165,11 @@ def _draw_ctx(cfg: RoundConfig) -> np.ndarray:
     raise ValueError(d)
 
 
+def draw_ctx_len(cfg: RoundConfig) -> np.ndarray:
+    """Context lengths of `cfg.batch` requests from the configuration's distribution (int32)."""
+    return _draw_ctx(cfg)
+
+
 def make_batch_meta(cfg: RoundConfig) -> BatchMeta:
     B, bs, g1 = cfg.batch, cfg.block_size, cfg.gamma + 1
     ctx = _draw_ctx(cfg)
