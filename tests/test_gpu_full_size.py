@@ -5,8 +5,9 @@ compute one by one: attention rows of sampled requests in sampled layers, whole
 slabs of the pool bit for bit, and the acceptance of every request.
 
 knee_b512 (the benchmark's workload) always runs at full size.  The two larger
-configs run at full context lengths, gamma and reassignment share with a reduced
-batch unless NSD_FULL_SIZE=1 (their single slabs are 11 and 19 GB on the host)."""
+configs run at full size too when the host has 96 GiB available (their single slabs are
+11 and 19 GB on the host; NSD_FULL_SIZE=1 / 0 forces either way); otherwise at full context
+lengths, gamma and reassignment share with a reduced batch."""
 import os
 
 import numpy as np
@@ -18,7 +19,22 @@ import workload as W
 from nsd_testlib import DeviceBatch, accept_compare, attn_mismatch, dev, host_u16, make_context
 
 pytestmark = pytest.mark.gpu
-FULL = os.environ.get("NSD_FULL_SIZE", "0") == "1"
+
+
+def _full_size() -> bool:
+    """NSD_FULL_SIZE=1 / 0 decides; unset: full size when the host has the memory for the larger slabs."""
+    env = os.environ.get("NSD_FULL_SIZE")
+    if env is not None:
+        return env == "1"
+    try:
+        import psutil
+
+        return psutil.virtual_memory().available >= 96 * 2 ** 30
+    except Exception:
+        return False
+
+
+FULL = _full_size()
 
 
 def _sample_requests(cfg, meta, n_random=3):
