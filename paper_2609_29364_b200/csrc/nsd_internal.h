@@ -18,8 +18,8 @@ struct __align__(16) AttnItem {
     int32_t chunk_idx;
     int32_t nchunks;
     int32_t src_off;     // first entry of the request's source blocks in the gather list, -1 = resident
-    int32_t ctx;         // the request's context length when the plan was made (tcgen05 path: saves a dependent load)
-    int32_t tbl_off;     // kv_indptr[req] when the plan was made (same)
+    int32_t ctx;         // the request's context length when the plan was made (saves the kernels a dependent load)
+    int32_t tbl_off;     // kv_indptr[req] when the plan was made (same); -1 = read kv_indptr[req] on the device
     int32_t pad[3];
 };
 static_assert(sizeof(AttnItem) == 48, "AttnItem is read as three 16-byte words");

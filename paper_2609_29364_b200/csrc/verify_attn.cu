@@ -145,10 +145,10 @@ verify_attn_kernel(const AttnLaunch a) {
     const AttnItem it = a.items[item_idx];
     const int r = it.req;
     const int gamma = a.gamma;
-    const int ctx = a.ctx_len[r];
+    const int ctx = it.ctx;                       // the plan's copy of ctx_len[r]: one dependent load less before the first tile
     const int n_total = ctx + gamma + 1;          // keys that exist after the append
     const int M = a.m_rows;
-    const int64_t table0 = a.kv_indptr[r];
+    const int64_t table0 = it.tbl_off >= 0 ? (int64_t)it.tbl_off : a.kv_indptr[r];
     const int n_blk = it.blk_end - it.blk_begin;
     const int n_tiles = (n_blk + KG - 1) / KG;
 
@@ -484,34 +484,65 @@ verify_attn_kernel(const AttnLaunch a) {
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    for (int e = tid; e < M * (D / 4); e += NT) {
-        const int m = e / (D / 4), d4 = e - m * (D / 4);
-        float mstar = -INFINITY;
+    // Thread = one 4-dim column of RB rows at a time: the RB rows' loads of a chunk are independent, so a merge costs
+    // about 2 * nchunks L2 round trips per row batch instead of per row.
+    constexpr int C4 = D / 4, RP = NT / C4, RB = 8;
+    static_assert(NT % C4 == 0, "threads cover whole rows of 4-dim columns");
+    const int d4 = tid % C4;
+    for (int mb = tid / C4; mb < M; mb += RP * RB) {
+        float mstar[RB];
+#pragma unroll
+        for (int k = 0; k < RB; ++k) mstar[k] = -INFINITY;
+        for (int c = 0; c < it.nchunks; ++c) {
+            const float* ml = a.part_ml + (((int64_t)it.part_base + c) * Hkv + head) * M * 2;
+#pragma unroll
+            for (int k = 0; k < RB; ++k) {
+                const int m = mb + k * RP;
+                if (m < M) mstar[k] = fmaxf(mstar[k], __ldcg(ml + m * 2));
+            }
+        }
+        float4 acc[RB];
+        float l[RB];
+#pragma unroll
+        for (int k = 0; k < RB; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f), l[k] = 0.f;
         for (int c = 0; c < it.nchunks; ++c) {
             const int64_t slot = ((int64_t)it.part_base + c) * Hkv + head;
-            mstar = fmaxf(mstar, __ldcg(a.part_ml + (slot * M + m) * 2));
+            float2 ml[RB];
+            float4 v[RB];
+#pragma unroll
+            for (int k = 0; k < RB; ++k) {
+                const int m = mb + k * RP;
+                ml[k] = make_float2(-INFINITY, 0.f);
+                v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (m < M) {
+                    ml[k] = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (slot * M + m) * 2));
+                    v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_acc + (slot * M + m) * D) + d4);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < RB; ++k) {
+                const float w = ml[k].x == -INFINITY ? 0.f : exp2f(ml[k].x - mstar[k]);
+                acc[k].x += w * v[k].x;
+                acc[k].y += w * v[k].y;
+                acc[k].z += w * v[k].z;
+                acc[k].w += w * v[k].w;
+                l[k] += w * ml[k].y;
+            }
         }
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float l = 0.f;
-        for (int c = 0; c < it.nchunks; ++c) {
-            const int64_t slot = ((int64_t)it.part_base + c) * Hkv + head;
-            const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (slot * M + m) * 2));
-            const float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mstar);
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_acc + (slot * M + m) * D) + d4);
-            acc.x += w * v.x;
-            acc.y += w * v.y;
-            acc.z += w * v.z;
-            acc.w += w * v.w;
-            l += w * ml.y;
+#pragma unroll
+        for (int k = 0; k < RB; ++k) {
+            const int m = mb + k * RP;
+            if (m < M) {
+                const float inv = 1.f / l[k];
+                const int i = m / G, h = m - i * G;
+                const int64_t orow = ((row_base + i) * Hq + head * G + h);
+                uint2 packed;
+                packed.x = pack_bf16(acc[k].x * inv, acc[k].y * inv);
+                packed.y = pack_bf16(acc[k].z * inv, acc[k].w * inv);
+                *reinterpret_cast<uint2*>(a.o + orow * D + d4 * 4) = packed;
+                if (a.lse && d4 == 0) a.lse[orow] = (mstar[k] + log2f(l[k])) * 0.6931471805599453f;
+            }
         }
-        const float inv = 1.f / l;
-        const int i = m / G, h = m - i * G;
-        const int64_t orow = ((row_base + i) * Hq + head * G + h);
-        uint2 packed;
-        packed.x = pack_bf16(acc.x * inv, acc.y * inv);
-        packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-        *reinterpret_cast<uint2*>(a.o + orow * D + d4 * 4) = packed;
-        if (a.lse && d4 == 0) a.lse[orow] = (mstar + log2f(l)) * 0.6931471805599453f;
     }
 }
 
@@ -543,7 +574,7 @@ cudaError_t attn_init() {
     if ((e = init_one<DD, WW, TT, KK, SS>()) != cudaSuccess) return e;
     NSD_ATTN_SHAPES(NSD_INIT, 64, kStagesD64)
     NSD_ATTN_SHAPES(NSD_INIT, 128, kStagesD128)
-    NSD_INIT(128, 1, 3, 16, 3) NSD_INIT(128, 1, 3, 32, 2) NSD_INIT(128, 1, 3, 32, 3)
+    NSD_INIT(128, 1, 3, 16, 3) NSD_INIT(128, 1, 3, 32, 2) NSD_INIT(128, 1, 3, 32, 3) NSD_INIT(128, 1, 3, 16, 8) NSD_INIT(128, 1, 3, 16, 6)
 #undef NSD_INIT
     return cudaSuccess;
 }
@@ -555,6 +586,8 @@ cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
     const int nw = (nt8 + 2) / 3, ntw = (nt8 + nw - 1) / nw;
     if (a.shape.D == 128 && nw == 1 && ntw == 3) {      // experiment knob: tile keys * 10 + ring depth
         if (a.tune_stages == 163) return launch_one<128, 1, 3, 16, 3>(a, stream);
+        if (a.tune_stages == 168) return launch_one<128, 1, 3, 16, 8>(a, stream);
+        if (a.tune_stages == 166) return launch_one<128, 1, 3, 16, 6>(a, stream);
         if (a.tune_stages == 322) return launch_one<128, 1, 3, 32, 2>(a, stream);
         if (a.tune_stages == 323) return launch_one<128, 1, 3, 32, 3>(a, stream);
     }
@@ -657,6 +690,8 @@ extern "C" nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_bl
             it.part_base = n > 1 ? slots : -1;
             it.chunk_idx = c;
             it.nchunks = (int32_t)n;
+            it.ctx = h_ctx_len[r];
+            it.tbl_off = -1;                              // this entry point has no host copy of kv_indptr
             items[n_items++] = it;
         }
         if (n > 1) slots += (int)n;
