@@ -34,9 +34,9 @@ import workload as W  # noqa: E402
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic byte of verify_attn_kernel, from the
-# ncu capture of the reduced case summarised in profiles/verify_attn_kernel_ncu.md (737.6 MB over 698.9 MB for one whole-batch pass); the
+# ncu capture of the reduced case summarised in profiles/verify_attn_kernel_ncu.md (709.4 MB over 698.9 MB for one whole-batch pass); the
 # full-size launch is too large to capture under the profiler, and traffic grows with the keys streamed.
-ATTN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.055
+ATTN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.015
 
 
 def parse_args():
