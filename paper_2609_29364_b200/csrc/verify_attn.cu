@@ -574,7 +574,7 @@ cudaError_t attn_init() {
     if ((e = init_one<DD, WW, TT, KK, SS>()) != cudaSuccess) return e;
     NSD_ATTN_SHAPES(NSD_INIT, 64, kStagesD64)
     NSD_ATTN_SHAPES(NSD_INIT, 128, kStagesD128)
-    NSD_INIT(128, 1, 3, 16, 3) NSD_INIT(128, 1, 3, 32, 2) NSD_INIT(128, 1, 3, 32, 3) NSD_INIT(128, 1, 3, 16, 8) NSD_INIT(128, 1, 3, 16, 6)
+    NSD_INIT(128, 1, 3, 16, 3) NSD_INIT(128, 1, 3, 32, 2) NSD_INIT(128, 1, 3, 32, 3)
 #undef NSD_INIT
     return cudaSuccess;
 }
@@ -586,8 +586,6 @@ cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
     const int nw = (nt8 + 2) / 3, ntw = (nt8 + nw - 1) / nw;
     if (a.shape.D == 128 && nw == 1 && ntw == 3) {      // experiment knob: tile keys * 10 + ring depth
         if (a.tune_stages == 163) return launch_one<128, 1, 3, 16, 3>(a, stream);
-        if (a.tune_stages == 168) return launch_one<128, 1, 3, 16, 8>(a, stream);
-        if (a.tune_stages == 166) return launch_one<128, 1, 3, 16, 6>(a, stream);
         if (a.tune_stages == 322) return launch_one<128, 1, 3, 32, 2>(a, stream);
         if (a.tune_stages == 323) return launch_one<128, 1, 3, 32, 3>(a, stream);
     }
