@@ -22,6 +22,7 @@ struct nsd_ctx {
     size_t ws_bytes;
     int32_t* d_status;       // [4]
     int32_t* d_counters;     // [max_batch * Hkv]
+    AcceptSplit accept_split; // scratch rows and counters for sharing a request among acceptance CTAs
     AttnItem* d_items_all;   // [max_items]
     AttnItem* d_items_split; // [max_items]  resident items then reassigned items
     float* d_part_ml;        // [part_slots * Hkv * Mmax * 2]
@@ -72,9 +73,9 @@ bool config_supported(const nsd_config* c) {
 }
 
 struct Layout {
-    size_t status, counters, items_all, items_split, part_ml, part_acc, total;
+    size_t status, counters, acc_counters, items_all, items_split, acc_scratch, part_ml, part_acc, total;
     int64_t max_items, part_slots;
-    int32_t m_max;
+    int32_t m_max, acc_rows;
 };
 
 Layout make_layout(const nsd_config* c) {
@@ -86,8 +87,11 @@ Layout make_layout(const nsd_config* c) {
     size_t off = 0;
     L.status = off;      off = align_up(off + 4 * sizeof(int32_t), 256);
     L.counters = off;    off = align_up(off + (size_t)c->max_batch * c->num_kv_heads * sizeof(int32_t), 256);
+    L.acc_rows = std::min<int32_t>(c->max_batch, 512);                   // requests that may be shared among acceptance CTAs
+    L.acc_counters = off; off = align_up(off + (size_t)L.acc_rows * sizeof(int32_t), 256);
     L.items_all = off;   off = align_up(off + (size_t)L.max_items * sizeof(AttnItem), 256);
     L.items_split = off; off = align_up(off + (size_t)L.max_items * sizeof(AttnItem), 256);
+    L.acc_scratch = off; off = align_up(off + (size_t)L.acc_rows * ((c->vocab_size + 127) / 128) * sizeof(double), 256);
     L.part_ml = off;     off = align_up(off + (size_t)L.part_slots * c->num_kv_heads * L.m_max * 2 * sizeof(float), 256);
     L.part_acc = off;    off = align_up(off + (size_t)L.part_slots * c->num_kv_heads * L.m_max * c->head_dim * sizeof(float), 256);
     L.total = off;
@@ -159,6 +163,8 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     ctx->d_items_all = reinterpret_cast<AttnItem*>(ctx->ws + L.items_all);
     ctx->d_items_split = reinterpret_cast<AttnItem*>(ctx->ws + L.items_split);
     ctx->d_part_ml = reinterpret_cast<float*>(ctx->ws + L.part_ml);
+    ctx->accept_split = AcceptSplit{reinterpret_cast<double*>(ctx->ws + L.acc_scratch), reinterpret_cast<int32_t*>(ctx->ws + L.acc_counters),
+                                    L.acc_rows, cfg->vocab_size, 0};
     ctx->d_part_acc = reinterpret_cast<float*>(ctx->ws + L.part_acc);
     ctx->max_items = L.max_items;
     ctx->part_slots = L.part_slots;
@@ -212,6 +218,7 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     ctx->tmaps.resize(cfg->num_slabs);
     ctx->tmap_slab.assign(cfg->num_slabs, nullptr);
     if ((e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device)) != cudaSuccess) return fail(e, "cudaDeviceGetAttribute");
+    ctx->accept_split.n_sms = ctx->n_sms;
     {
         const char* path = getenv("NSD_ATTN_PATH");          // "mma" or "tcgen05"; default below
         ctx->attn_path = path ? (strcmp(path, "tcgen05") == 0) : 0;
@@ -493,7 +500,7 @@ nsd_status nsd_spec_accept(nsd_ctx* ctx, const float* p, const float* q, const i
     if (!p || !q || !draft_tok || !u_acc || !u_smp || !acc_len || !out_tok) return NSD_ERR_INVALID_ARG;
     if ((new_ctx_len != nullptr) && !ctx_len) return NSD_ERR_INVALID_ARG;
     NSD_CUDA(ctx, launch_accept(p, q, draft_tok, u_acc, u_smp, batch, gamma, vocab, ctx_len, acc_len, out_tok,
-                                new_ctx_len, ctx->d_status, static_cast<cudaStream_t>(stream)));
+                                new_ctx_len, ctx->d_status, ctx->accept_split, static_cast<cudaStream_t>(stream)));
     ctx->launches++;
     return NSD_OK;
 }
@@ -621,7 +628,7 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
         NSD_CUDA(ctx, cudaStreamWaitEvent(st, hook->inputs_ready, 0));
     }
     NSD_CUDA(ctx, launch_accept(a->p, a->q_draft, a->draft_tok, a->u_acc, a->u_smp, batch, gamma, ctx->cfg.vocab_size,
-                                a->ctx_len, a->acc_len, a->out_tok, a->new_ctx_len, ctx->d_status, st));
+                                a->ctx_len, a->acc_len, a->out_tok, a->new_ctx_len, ctx->d_status, ctx->accept_split, st));
     ctx->launches++;
     if (hook) NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down_done, 0));      // the caller's stream covers the read-back
     return NSD_OK;

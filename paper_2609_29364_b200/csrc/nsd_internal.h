@@ -80,10 +80,17 @@ bool attn_umma_supported(const AttnLaunch& a);
 cudaError_t launch_attn_umma(const AttnLaunch& a, cudaStream_t stream, int n_sms);
 bool make_kv_tensor_map(CUtensorMap* map, const void* slab, const Shape& s);
 cudaError_t attn_init();          // opt in to large dynamic shared memory, once per process
+// Scratch for sharing one request among several acceptance CTAs (small batches): one row of segment sums and one
+// arrival counter (zero between launches) per request.
+struct AcceptSplit {
+    double* scratch;      // [rows_cap][ceil(vocab_cap / 128)]
+    int32_t* counters;    // [rows_cap]
+    int32_t rows_cap, vocab_cap, n_sms;
+};
 cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
                           const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int32_t* ctx_len,
                           int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
-                          cudaStream_t stream);
+                          const AcceptSplit& split, cudaStream_t stream);
 
 cudaError_t launch_accept_logits(const void* logits, int32_t logits_bf16, float temperature, const float* q,
                                  const int32_t* draft_tok, const float* u_acc, const float* u_smp, int32_t batch,

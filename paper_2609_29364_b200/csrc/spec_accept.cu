@@ -7,7 +7,11 @@
 // the whole CTA then sweeps ONLY the one vocabulary row pair that the draw needs
 // (not all gamma+1), keeping one partial sum per 128-token segment in shared
 // memory; the segment that holds the draw is found from the segment prefix and
-// re-read (an L2 hit) to finish inside it.  All compares and sums are fp64 on the
+// re-read (an L2 hit) to finish inside it.  When the batch is too small to fill
+// the machine, `split` CTAs share a request: each sweeps its slice of the segments
+// into a scratch row, and the last one to finish (atomic counter, nobody waits)
+// collects the row and draws; segment sums, prefix and draw are the same numbers
+// in the same order either way.  All compares and sums are fp64 on the
 // fp32 inputs, the residual is a single fp32 subtraction, so decisions agree
 // with a sequential fp64 evaluation except within rounding of a CDF boundary.
 // Compile without fast-math: IEEE division and no flush-to-zero are required.
@@ -36,12 +40,13 @@ __global__ void __launch_bounds__(kAcceptThreads)
 spec_accept_kernel(const float* __restrict__ p, const float* __restrict__ q, const int32_t* __restrict__ draft_tok,
                    const float* __restrict__ u_acc, const float* __restrict__ u_smp, int32_t gamma, int32_t vocab,
                    const int32_t* __restrict__ ctx_len, int32_t* __restrict__ acc_len, int32_t* __restrict__ out_tok,
-                   int32_t* __restrict__ new_ctx_len, int32_t* __restrict__ status) {
+                   int32_t* __restrict__ new_ctx_len, int32_t* __restrict__ status, int32_t split,
+                   double* __restrict__ seg_scratch, int32_t* __restrict__ seg_counters) {
     extern __shared__ double seg_sum[];          // [n_seg] segment sums, then exclusive prefixes
-    __shared__ int s_n, s_found_seg, s_token;
+    __shared__ int s_n, s_found_seg, s_token, s_last;
     __shared__ double s_total;
 
-    const int r = blockIdx.x;
+    const int r = blockIdx.x / split, part = blockIdx.x - r * split;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_warps = kAcceptThreads / 32;
     const int n_seg = (vocab + kSeg - 1) / kSeg;
@@ -75,9 +80,9 @@ spec_accept_kernel(const float* __restrict__ p, const float* __restrict__ q, con
     bool residual = n < gamma;
     const bool vec_ok = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(q)) % 16 == 0);
 
-    for (int attempt = 0; attempt < 2; ++attempt) {
-        // ---- pass 1: one sum per segment
-        for (int s = warp; s < n_seg; s += n_warps) {
+    // ---- pass 1: one sum per segment of [s_begin, s_end), into shared memory or into the request's scratch row
+    auto sweep = [&](int s_begin, int s_end, double* dst) {
+        for (int s = s_begin + warp; s < s_end; s += n_warps) {
             const int k0 = s * kSeg + lane * 4;
             double acc = 0.0;
             if (vec_ok) {
@@ -96,10 +101,11 @@ spec_accept_kernel(const float* __restrict__ p, const float* __restrict__ q, con
                     if (k0 + j < vocab) acc += (double)weight(prow[k0 + j], residual ? qrow[k0 + j] : 0.f, residual);
             }
             acc = warp_sum(acc);
-            if (lane == 0) seg_sum[s] = acc;
+            if (lane == 0) dst[s] = acc;
         }
-        __syncthreads();
-        // ---- exclusive prefix over segments (warp 0, lanes own consecutive runs)
+    };
+    // ---- exclusive prefix over segments (warp 0, lanes own consecutive runs)
+    auto prefix = [&]() {
         if (warp == 0) {
             const int per = (n_seg + 31) / 32;
             const int b = lane * per, e = min(b + per, n_seg);
@@ -124,12 +130,36 @@ spec_accept_kernel(const float* __restrict__ p, const float* __restrict__ q, con
             }
         }
         __syncthreads();
-        if (residual && s_total == 0.0) {       // empty residual: draw from the target row instead
-            residual = false;
-            __syncthreads();
-            continue;
+    };
+
+    if (split == 1) {
+        sweep(0, n_seg, seg_sum);
+    } else {
+        // this CTA's slice goes to the scratch row; whoever arrives last owns the rest of the work
+        double* row = seg_scratch + (int64_t)r * n_seg;
+        const int per = (n_seg + split - 1) / split;
+        sweep(part * per, min((part + 1) * per, n_seg), row);
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            const int old = atomicAdd(seg_counters + r, 1);
+            const int last = old == split - 1;
+            if (last) seg_counters[r] = 0;           // ready for the next launch
+            s_last = last;
         }
-        break;
+        __syncthreads();
+        if (!s_last) return;
+        __threadfence();
+        for (int s = tid; s < n_seg; s += kAcceptThreads) seg_sum[s] = __ldcg(row + s);
+    }
+    __syncthreads();
+    prefix();
+    if (residual && s_total == 0.0) {           // empty residual: draw from the target row instead
+        residual = false;
+        __syncthreads();
+        sweep(0, n_seg, seg_sum);
+        __syncthreads();
+        prefix();
     }
 
     const double total = s_total;
@@ -198,7 +228,7 @@ spec_accept_kernel(const float* __restrict__ p, const float* __restrict__ q, con
 cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
                           const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int32_t* ctx_len,
                           int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
-                          cudaStream_t stream) {
+                          const AcceptSplit& sp, cudaStream_t stream) {
     if (batch <= 0) return cudaSuccess;
     const int n_seg = (vocab + kSeg - 1) / kSeg;
     const size_t smem = (size_t)(n_seg + 1) * sizeof(double);
@@ -206,8 +236,17 @@ cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_t
         cudaError_t e = cudaFuncSetAttribute(spec_accept_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    spec_accept_kernel<<<batch, kAcceptThreads, smem, stream>>>(p, q, draft_tok, u_acc, u_smp, gamma, vocab, ctx_len,
-                                                              acc_len, out_tok, new_ctx_len, status);
+    // Several CTAs per request while that still leaves the machine under two CTAs per SM, the slices at least
+    // eight passes of a CTA long, and the scratch rows large enough.
+    int split = 1;
+    if (sp.scratch && sp.counters && batch <= sp.rows_cap && vocab <= sp.vocab_cap && sp.n_sms > 0) {
+        split = (2 * sp.n_sms) / batch;
+        split = split < 1 ? 1 : (split > 8 ? 8 : split);
+        while (split > 1 && n_seg / split < 8 * (kAcceptThreads / 32)) --split;
+    }
+    spec_accept_kernel<<<batch * split, kAcceptThreads, smem, stream>>>(p, q, draft_tok, u_acc, u_smp, gamma, vocab, ctx_len,
+                                                                      acc_len, out_tok, new_ctx_len, status, split,
+                                                                      sp.scratch, sp.counters);
     return cudaGetLastError();
 }
 

@@ -86,6 +86,33 @@ def test_empty_residual_and_all_zero_rows():
     assert acc.tolist() == [0, 1, 0] and out[2].tolist() == [-1, -1]
 
 
+@pytest.mark.parametrize("batch", [1, 3, 37, 150])
+def test_small_batches_share_a_request_among_ctas(batch):
+    """Below two CTAs per SM the kernel gives a request to several CTAs (2..8 here, 1 at batch 150 and
+    above): same lengths, same tokens as the oracle, twice in a row (the arrival counters must be back
+    at zero), including a request whose residual is empty and one whose rows are all zero."""
+    V, g = 70000, 3
+    cfg = W.RoundConfig("accsplit", batch=batch, gamma=g, num_layers=1, num_q_heads=8, num_kv_heads=2, head_dim=64,
+                        block_size=16, vocab=V, ctx_dist=("fixed", [1] * batch), frac_reassigned=0.0, noise_var=1.0, seed=77 + batch)
+    p, q, tok, ua, us = W.accept_inputs(cfg)
+    q[0, 0] = 1.0 / V
+    p[0, 0] = 0.25 / V                                       # p <= q everywhere at the first position of request 0 ...
+    ua[0, 0] = 0.9                                           # ... which is rejected: the draw falls back to the target row
+    if batch > 2:
+        p[2] = 0.0                                           # nothing to draw from at all -> token -1
+    ctx = _ctx(V, batch, g)
+    acc_r, out_r, _ = oracle.spec_accept(p, q, tok, ua, us)
+    for _ in range(2):
+        acc_g, out_g, _ = run_accept_gpu(ctx, p, q, tok, ua, us)
+        rc, bad = ctx.nsd_get_status()
+        assert rc == 0, (rc, bad)
+        rep = accept_compare(p, q, tok, ua, us, acc_g, out_g, acc_r, out_r)
+        assert rep["len_exact"] == batch, rep
+    assert acc_r[0] == 0 and out_g[0, 0] >= 0
+    if batch > 2:
+        assert out_g[2].tolist().count(-1) >= 1
+
+
 def test_out_of_vocab_draft_token_is_reported_and_rejected():
     V = 64
     rng = np.random.default_rng(0)
