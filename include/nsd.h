@@ -26,6 +26,11 @@
  *    failing call launches nothing.  Device-side index checks (block ids read
  *    from device tables) never fault: a bad id is replaced by block 0, the
  *    event is recorded in a status word, and nsd_get_status reports it.
+ *  - A context is one worker: its workspace holds the plan, the split-KV partials,
+ *    the acceptance scratch and the status word, so calls on ONE context must not
+ *    overlap on the GPU (enqueue them on one stream, or order the streams with
+ *    events); different contexts are independent.  nsd_create also owns a copy
+ *    stream and a read-back stream used only by nsd_verify_round_host.
  *  - bf16 tensors are raw 16-bit patterns.  Compiled for sm_100a only.
  *
  * KV pool layout (bf16):
