@@ -27,10 +27,14 @@
  *    from device tables) never fault: a bad id is replaced by block 0, the
  *    event is recorded in a status word, and nsd_get_status reports it.
  *  - A context is one worker: its workspace holds the plan, the split-KV partials,
- *    the acceptance scratch and the status word, so calls on ONE context must not
- *    overlap on the GPU (enqueue them on one stream, or order the streams with
- *    events); different contexts are independent.  nsd_create also owns a copy
- *    stream and a read-back stream used only by nsd_verify_round_host.
+ *    the acceptance scratch and the status word.  nsd_verify_attn, nsd_spec_accept,
+ *    nsd_spec_accept_logits and nsd_verify_round(_host) on ONE context must not
+ *    overlap one another on the GPU (enqueue them on one stream, or order the streams
+ *    with events).  nsd_kv_prepare and nsd_kv_commit touch only the pool and the
+ *    status word and may run on other streams beside them, as long as the caller
+ *    orders the accesses to the same blocks.  Different contexts are independent.
+ *    nsd_create also owns a copy stream and a read-back stream used only by
+ *    nsd_verify_round_host.
  *  - bf16 tensors are raw 16-bit patterns.  Compiled for sm_100a only.
  *
  * KV pool layout (bf16):
