@@ -47,7 +47,7 @@ struct nsd_ctx {
     std::vector<CUtensorMap> tmaps;
     std::vector<const void*> tmap_slab;
     int n_sms;
-    int attn_path;             // 0 = mma.sync kernel, 1 = tcgen05 kernel where it applies
+    int attn_path;             // 0 = mma.sync kernel fed by cp.async, 1 = tcgen05 kernel where it applies, 2 = mma.sync fed by TMA where faster (default)
     int64_t launches;
     char err[256];
 };
@@ -220,8 +220,10 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     if ((e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device)) != cudaSuccess) return fail(e, "cudaDeviceGetAttribute");
     ctx->accept_split.n_sms = ctx->n_sms;
     {
-        const char* path = getenv("NSD_ATTN_PATH");          // "mma" or "tcgen05"; default below
-        ctx->attn_path = path ? (strcmp(path, "tcgen05") == 0) : 0;
+        // Default: the mma.sync kernel with its K/V tiles fetched by tensor copies where that is the faster feed
+        // (cp.async otherwise).  NSD_ATTN_PATH=mma forces cp.async everywhere, =tcgen05 selects the tcgen05 engine.
+        const char* path = getenv("NSD_ATTN_PATH");
+        ctx->attn_path = !path ? 2 : (strcmp(path, "tcgen05") == 0 ? 1 : (strcmp(path, "mma") == 0 ? 0 : 2));
     }
     *out = ctx;
     return NSD_OK;
@@ -455,7 +457,7 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
     else if (subset == 1) { a.items = ctx->d_items_split; a.n_items = ctx->n_res; }
     else { a.items = ctx->d_items_split + ctx->n_res; a.n_items = ctx->n_mig_items; }
     if (a.n_items == 0) return NSD_OK;
-    if (ctx->attn_path == 1 && !fuse && ctx->cfg.head_dim == 128) {
+    if (ctx->attn_path != 0 && !fuse && ctx->cfg.head_dim == 128) {
         const int slab = layer % ctx->cfg.num_slabs;
         if (ctx->tmap_slab[slab] != a.pool_slab) {
             ctx->tmap_slab[slab] = make_kv_tensor_map(&ctx->tmaps[slab], a.pool_slab, ctx->shape) ? a.pool_slab : nullptr;
@@ -464,7 +466,8 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
             a.tmap = ctx->tmaps[slab];
             a.tmap_valid = 1;
         }
-        if (attn_umma_supported(a)) {
+        a.tma_feed = ctx->attn_path == 2;
+        if (ctx->attn_path == 1 && attn_umma_supported(a)) {
             NSD_CUDA(ctx, launch_attn_umma(a, st, ctx->n_sms));
             ctx->launches++;
             return NSD_OK;

@@ -23,9 +23,15 @@
 // chunks and orders the chunk items longest first; the grid is one CTA per
 // (item, kv head), scheduled by the hardware in that order.  A CTA has one warp per
 // group of up to three 8-row tiles (one warp at gamma 4).  K/V tiles of one pool block
-// stream global -> shared through a cp.async ring whose rows are padded by 16 bytes
-// (conflict-free ldmatrix, every address a per-thread constant plus a compile-time
-// offset; the ring loop is unrolled by stage).  A request with one chunk writes bf16
+// stream global -> shared through a four-stage ring (every fragment address a per-thread
+// constant plus a compile-time offset; the ring loop is unrolled by stage), fed in one of
+// two ways.  Tensor copies (the default where the shape is bound by HBM, up to four row
+// tiles): four cp.async.bulk.tensor boxes of 16 keys x 64 dims per tile, issued by four
+// lanes, land in the 128-byte-swizzled layout and complete on the stage's mbarrier; the
+// consumer spends one wait and five instructions per tile on the feed instead of sixteen
+// cp.async per lane, which is worth 4-6 % under the power cap.  cp.async (five or six row
+// tiles, head_dim 64, gather-through, the allocation-free entry): rows padded by 16 bytes
+// for conflict-free ldmatrix.  A request with one chunk writes bf16
 // output directly; otherwise the CTA stores its unnormalised fp32 partial (max, sum,
 // acc) and the LAST CTA to finish that (request, head) -- decided by an atomic
 // counter, nobody waits -- merges all partials in chunk order and writes the output.
@@ -96,6 +102,32 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// ---- TMA-fed variant: mbarrier and tensor-copy helpers --------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded: gives up after ~2^20 hardware wait slices (seconds); the caller then records STATUS_TIMEOUT and leaves.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < (1u << 20); ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity), "r"(2000u)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+                 : "memory");
+}
+
 // Shared-memory tiles are [rows][D] bf16 with every row padded by 16 bytes: eight
 // consecutive rows then start 16 bytes apart modulo 128, so the eight row reads of
 // one ldmatrix phase hit distinct banks.
@@ -105,21 +137,25 @@ struct Tile {
     static constexpr int kBytes = TK * kPitch;                      // K (or V) of one stage
 };
 
-// TK = keys per pipeline stage (one or two pool blocks), kStages = ring depth.
-template <int D, int TK, int kStages, int ROWS>
+// TK = keys per pipeline stage (one or two pool blocks), kStages = ring depth.  The TMA-fed variant keeps the
+// tiles unpadded in the 128-byte-swizzled layout the tensor copy writes: [K lo | K hi | V lo | V hi], each
+// [TK keys][64 dims].
+template <int D, int TK, int kStages, int ROWS, bool TMA = false>
 struct Smem {
-    static constexpr int kStageBytes = 2 * Tile<D, TK>::kBytes;     // K then V
+    static constexpr int kStageBytes = TMA ? 2 * TK * D * 2 : 2 * Tile<D, TK>::kBytes;     // K then V
     static constexpr int kMaxChunkBlocks = 256;                     // ids to read from + ids to write to
     static constexpr int kOutPitch = D + 4;                         // floats per staged output row
     static constexpr int kOutBytes = (ROWS * kOutPitch + 2 * ROWS) * 4;   // output staging reuses the ring
     static constexpr int kRingBytes = kStages * kStageBytes > kOutBytes ? kStages * kStageBytes : (kOutBytes + 15) / 16 * 16;
-    static constexpr int kBytes = kRingBytes + 2 * kMaxChunkBlocks * 4;
+    static constexpr int kBytes = kRingBytes + 2 * kMaxChunkBlocks * 4 + (TMA ? 1024 : 0);
 };
 
-// NW warps, each serving NTW tiles of 8 query rows; rows m >= M are zero padding.
-template <int D, int NW, int NTW, int TK, int kStages>
+// NW warps, each serving NTW tiles of 8 query rows; rows m >= M are zero padding.  TMA = the K/V tiles arrive by
+// cp.async.bulk.tensor boxes (one warp, head_dim 128, one pool block per stage, no gather-through) instead of cp.async.
+template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false>
 __global__ void __launch_bounds__(NW * 32)
-verify_attn_kernel(const AttnLaunch a) {
+verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
+    static_assert(!TMA || (D == 128 && TK == 16), "the TMA-fed variant covers head_dim 128 with one pool block per stage");
     constexpr int KG = TK / 16;                   // 16-key groups (= pool blocks) per tile
     constexpr int NT = NW * 32;                   // threads
     constexpr int CPR = D / 8;                    // 16-byte pieces per row
@@ -128,15 +164,19 @@ verify_attn_kernel(const AttnLaunch a) {
     constexpr int PITCH = Tile<D, TK>::kPitch;
     constexpr int TILE = Tile<D, TK>::kBytes;
     constexpr int ROWS_PAD = NW * NTW * 8;        // query rows incl. padding
-    using SM = Smem<D, TK, kStages, ROWS_PAD>;
+    using SM = Smem<D, TK, kStages, ROWS_PAD, TMA>;
     constexpr int STAGE = SM::kStageBytes;
     constexpr int OPITCH = SM::kOutPitch;
     constexpr int ROWS_PER_STEP = NT / CPR;       // rows one pass of all threads covers in a block copy
     constexpr int COPY_STEPS = (kBlockSize + ROWS_PER_STEP - 1) / ROWS_PER_STEP;
     static_assert(NT % CPR == 0, "a copy pass covers whole rows");
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    // the swizzled tiles of the TMA-fed variant must start on a 1024-byte boundary (its size carries the slack)
+    unsigned char* const smem = TMA ? reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023) : smem_raw;
     int32_t* blk_s = reinterpret_cast<int32_t*>(smem + SM::kRingBytes);
     __shared__ int s_last;
+    __shared__ __align__(8) uint64_t full_bar[kStages];      // TMA-fed variant: a stage's bytes have landed
+    __shared__ volatile int s_timeout;                       // ... or never did
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int Hkv = a.shape.Hkv, Hq = a.shape.Hq, G = Hq / Hkv;
@@ -154,7 +194,7 @@ verify_attn_kernel(const AttnLaunch a) {
 
     // Gather-through: a reassigned request streams its committed KV from the source blocks and writes it,
     // with the new tokens, to its destination blocks on the way (uniform per CTA).
-    const bool fused = a.fuse != 0 && it.src_off >= 0;
+    const bool fused = !TMA && a.fuse != 0 && it.src_off >= 0;
     const int n_src = (ctx + kBlockSize - 1) / kBlockSize;       // blocks that hold committed KV
     int32_t* dst_s = blk_s + SM::kMaxChunkBlocks;
 
@@ -181,7 +221,12 @@ verify_attn_kernel(const AttnLaunch a) {
         }
         blk_s[i] = b;
     }
-    __syncthreads();                              // blk_s visible before tiles are issued
+    if (TMA && tid == 0) {
+        s_timeout = 0;
+        for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&full_bar[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();                              // blk_s (and the barriers) visible before tiles are issued
 
     // ---- per-thread constants of the copy and of the fragment loads
     const uint32_t smem0 = smem_u32(smem);
@@ -196,9 +241,31 @@ verify_attn_kernel(const AttnLaunch a) {
     // V^T as A operand (16 dims x 16 keys), read transposed: a0 = keys 0-7 x dims 0-7, a1 = keys 0-7 x dims 8-15,
     // a2 = keys 8-15 x dims 0-7, a3 = keys 8-15 x dims 8-15
     const uint32_t v_frag = smem0 + TILE + ((mi >> 1) * 8 + (lane & 7)) * PITCH + (mi & 1) * 16;   // + stage, key group, dm
+    // TMA-fed variant: rows are 128 bytes and the 16-byte chunk c of row r sits at chunk c ^ (r & 7).  A fragment
+    // load of k-step kk (or dim tile dm) reads chunk 2 * (kk & 3) + h of half kk >> 2, h = the lane's matrix column:
+    // (2a + h) ^ x = 2a ^ (h ^ x), so four per-lane addresses cover every step with compile-time offsets on top.
+    uint32_t k_sw[4], v_sw[4];
+#pragma unroll
+    for (int a2 = 0; a2 < 4; ++a2) {
+        k_sw[a2] = smem0 + ((mi & 1) * 8 + (lane & 7)) * 128 + (((2 * a2) ^ ((mi >> 1) ^ (lane & 7))) << 4);
+        v_sw[a2] = smem0 + ((mi >> 1) * 8 + (lane & 7)) * 128 + (((2 * a2) ^ ((mi & 1) ^ (lane & 7))) << 4);
+    }
 
     // Issues the copy of tile t (KG pool blocks, K and V of this head) into `stage`.
     auto issue_tile = [&](int t, int stage) {
+        if constexpr (TMA) {
+            // four boxes of 16 keys x 64 dims (K lo, K hi, V lo, V hi), one per lane, completing on the stage's barrier
+            if (t < n_tiles && warp == 0) {
+                const uint32_t bar = smem_u32(&full_bar[stage]);
+                if (lane == 0) mbar_expect_tx(bar, STAGE);
+                __syncwarp();
+                if (lane < 4) {
+                    const int32_t row = ((blk_s[t] * 2 + (lane >> 1)) * Hkv + head) * kBlockSize;
+                    tma_load_2d(smem0 + stage * STAGE + lane * 2048, &a.tmap, (lane & 1) * 64, row, bar);
+                }
+            }
+            return;
+        }
         if (t < n_tiles) {
 #pragma unroll
             for (int half = 0; half < KG; ++half) {
@@ -264,9 +331,19 @@ verify_attn_kernel(const AttnLaunch a) {
     const int key0_chunk = it.blk_begin * kBlockSize;
     // One tile: wait for its copy, refill the stage freed by the previous tile, S^T = K Q^T,
     // online softmax, O^T += V^T P^T.  `stage` is a compile-time constant at every call site.
+    bool timed_out = false;                           // TMA-fed variant only: a stage never landed
     auto process_tile = [&](int t, int stage) {
-        cp_async_wait<kStages - 2>();
-        __syncthreads();
+        if constexpr (TMA) {
+            if (!mbar_wait(smem_u32(&full_bar[stage]), (uint32_t)((t / kStages) & 1))) s_timeout = 1;
+            __syncthreads();                          // every thread is done with tile t - 1, whose stage is refilled next
+            if (s_timeout) {                          // the same answer for every thread of the CTA
+                timed_out = true;
+                return;
+            }
+        } else {
+            cp_async_wait<kStages - 2>();
+            __syncthreads();
+        }
         issue_tile(t + kStages - 1, (stage + kStages - 1) % kStages);
         const int key0 = key0_chunk + t * TK;
         const bool need_mask = key0 + TK > ctx + 1;   // some key of the tile is hidden from some row
@@ -302,10 +379,18 @@ verify_attn_kernel(const AttnLaunch a) {
             __syncthreads();                                  // the copy has read the tile before anything zeroes it
         }
         if (key0 + TK > n_total) {                    // slots that hold no token: zero their V rows
-            unsigned char* vs = smem + stage * STAGE + TILE;
-            for (int c = tid; c < TK * CPR; c += NT) {
-                const int row = c / CPR, ch = c - row * CPR;
-                if (key0 + row >= n_total) *reinterpret_cast<int4*>(vs + row * PITCH + ch * 16) = make_int4(0, 0, 0, 0);
+            if constexpr (TMA) {
+                unsigned char* vs = smem + stage * STAGE + 4096;      // V lo, V hi: [16 keys][128 bytes] each
+                for (int c = tid; c < TK * 16; c += NT) {
+                    const int row = c >> 4, ch = c & 15;
+                    if (key0 + row >= n_total) *reinterpret_cast<int4*>(vs + (ch >> 3) * 2048 + row * 128 + (ch & 7) * 16) = make_int4(0, 0, 0, 0);
+                }
+            } else {
+                unsigned char* vs = smem + stage * STAGE + TILE;
+                for (int c = tid; c < TK * CPR; c += NT) {
+                    const int row = c / CPR, ch = c - row * CPR;
+                    if (key0 + row >= n_total) *reinterpret_cast<int4*>(vs + row * PITCH + ch * 16) = make_int4(0, 0, 0, 0);
+                }
             }
             __syncthreads();
         }
@@ -321,7 +406,8 @@ verify_attn_kernel(const AttnLaunch a) {
 #pragma unroll
             for (int kg = 0; kg < KG; ++kg) {
                 uint32_t kf[4];
-                ldmatrix_x4(kf, k_frag + stage * STAGE + kg * (16 * PITCH) + kk * 32);
+                if constexpr (TMA) ldmatrix_x4(kf, k_sw[kk & 3] + stage * STAGE + (kk >> 2) * 2048);
+                else ldmatrix_x4(kf, k_frag + stage * STAGE + kg * (16 * PITCH) + kk * 32);
 #pragma unroll
                 for (int j = 0; j < NTW; ++j) mma_bf16(sT[kg][j], kf, qb[kk][j][0], qb[kk][j][1]);
             }
@@ -394,17 +480,22 @@ verify_attn_kernel(const AttnLaunch a) {
 #pragma unroll
             for (int dm = 0; dm < DM; ++dm) {
                 uint32_t vf[4];
-                ldmatrix_x4_trans(vf, v_frag + stage * STAGE + kg * (16 * PITCH) + dm * 32);
+                if constexpr (TMA) ldmatrix_x4_trans(vf, v_sw[dm & 3] + stage * STAGE + 4096 + (dm >> 2) * 2048);
+                else ldmatrix_x4_trans(vf, v_frag + stage * STAGE + kg * (16 * PITCH) + dm * 32);
 #pragma unroll
                 for (int j = 0; j < NTW; ++j) mma_bf16(oT[dm][j], vf, pb[kg][j][0], pb[kg][j][1]);
             }
         }
     };
 
-    for (int t = 0; t < n_tiles; t += kStages) {
+    for (int t = 0; t < n_tiles && !timed_out; t += kStages) {
 #pragma unroll
         for (int s = 0; s < kStages; ++s)
-            if (t + s < n_tiles) process_tile(t + s, s);
+            if (t + s < n_tiles && !timed_out) process_tile(t + s, s);
+    }
+    if (timed_out) {                                      // nothing is written for this item; the status word says why
+        if (tid == 0) atomicOr(a.status, STATUS_TIMEOUT);
+        return;
     }
     cp_async_wait<0>();
     __syncthreads();                                      // the ring is free: reuse it to stage the output
@@ -546,17 +637,17 @@ verify_attn_kernel(const AttnLaunch a) {
     }
 }
 
-template <int D, int NW, int NTW, int TK, int kStages>
+template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false>
 cudaError_t launch_one(const AttnLaunch& a, cudaStream_t stream) {
     const int64_t grid = (int64_t)a.n_items * a.shape.Hkv;
-    verify_attn_kernel<D, NW, NTW, TK, kStages><<<(unsigned)grid, NW * 32, Smem<D, TK, kStages, NW * NTW * 8>::kBytes, stream>>>(a);
+    verify_attn_kernel<D, NW, NTW, TK, kStages, TMA><<<(unsigned)grid, NW * 32, Smem<D, TK, kStages, NW * NTW * 8, TMA>::kBytes, stream>>>(a);
     return cudaGetLastError();
 }
 
-template <int D, int NW, int NTW, int TK, int kStages>
+template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false>
 cudaError_t init_one() {
-    return cudaFuncSetAttribute(verify_attn_kernel<D, NW, NTW, TK, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                Smem<D, TK, kStages, NW * NTW * 8>::kBytes);
+    return cudaFuncSetAttribute(verify_attn_kernel<D, NW, NTW, TK, kStages, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                Smem<D, TK, kStages, NW * NTW * 8, TMA>::kBytes);
 }
 
 // One pool block per stage and a deeper ring gave the most resident warps per SM at the same bytes in flight.
@@ -575,6 +666,10 @@ cudaError_t attn_init() {
     NSD_ATTN_SHAPES(NSD_INIT, 64, kStagesD64)
     NSD_ATTN_SHAPES(NSD_INIT, 128, kStagesD128)
     NSD_INIT(128, 1, 3, 16, 3) NSD_INIT(128, 1, 3, 32, 2) NSD_INIT(128, 1, 3, 32, 3)
+#define NSD_INIT_TMA(DD, WW, TT, KK, SS) \
+    if ((e = init_one<DD, WW, TT, KK, SS, true>()) != cudaSuccess) return e;
+    NSD_ATTN_SHAPES(NSD_INIT_TMA, 128, kStagesD128)
+#undef NSD_INIT_TMA
 #undef NSD_INIT
     return cudaSuccess;
 }
@@ -584,6 +679,15 @@ cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
     const int nt8 = (a.m_rows + 7) / 8;                  // row tiles needed
     if (nt8 < 1 || nt8 > 8) return cudaErrorInvalidValue;
     const int nw = (nt8 + 2) / 3, ntw = (nt8 + nw - 1) / nw;
+    // K/V tiles by tensor copies where that measured faster: the shapes that are bound by HBM (up to 32 stacked rows:
+    // +4-6 % at 20-24 rows, +3 % at 28-32).  The five- and six-row-tile shapes are bound by the tensor pipe and by
+    // shared-memory reads and ran 8-25 % slower fed this way, so they stay on cp.async.
+    if (a.tma_feed && a.tmap_valid && !a.fuse && a.shape.D == 128 && (nw == 1 || (nw == 2 && ntw == 2))) {
+#define NSD_TMA_CASE(DD, WW, TT, KK, SS) \
+        if (nw == WW && ntw == TT) return launch_one<DD, WW, TT, KK, SS, true>(a, stream);
+        NSD_ATTN_SHAPES(NSD_TMA_CASE, 128, kStagesD128)
+#undef NSD_TMA_CASE
+    }
     if (a.shape.D == 128 && nw == 1 && ntw == 3) {      // experiment knob: tile keys * 10 + ring depth
         if (a.tune_stages == 163) return launch_one<128, 1, 3, 16, 3>(a, stream);
         if (a.tune_stages == 322) return launch_one<128, 1, 3, 32, 2>(a, stream);
