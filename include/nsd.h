@@ -8,10 +8,11 @@
  *   2. nsd_verify_attn  ragged paged grouped-query attention, gamma+1 causal
  *                       query rows per request (anchor + gamma proposals);
  *   3. nsd_spec_accept  speculative acceptance / residual resampling / bonus.
- * nsd_verify_round enqueues all three for every layer, with the preparation on
- * a side stream that overlaps attention (Section 4: Run(B_k) || Prepare(B_k+1),
- * here inside one batch: attention over resident requests || copy of the
- * reassigned ones).
+ * nsd_verify_round enqueues all three for every layer, with the block copies on
+ * a side stream that runs ahead of attention (Section 4: Run(B_k) || Prepare(B_k+1),
+ * here layer by layer inside one batch: the copy of layer l+1 is under way while
+ * layer l attends; only the first layer overlaps its own copy, by attending its
+ * resident requests first).
  *
  * Conventions
  *  - Every function returns nsd_status; NSD_OK = 0.  Nothing throws.
@@ -280,13 +281,16 @@ typedef struct {
 
 /*
  * One whole verification round (every step above, every logical layer),
- * enqueued with the preparation overlapped behind attention: per layer the
- * side stream gathers and appends the reassigned requests while `stream`
- * appends and attends the resident ones, then waits for the layer's copy event
- * (the KVReady condition of Eq. (F.3)) and attends the reassigned ones;
- * acceptance follows the last layer.  With num_slabs < num_layers the gather of
- * layer l also waits for attention of layer l - num_slabs.  Needs a plan for
- * this batch.  Returns after enqueue; `stream` carries the completion.
+ * enqueued with the preparation overlapped behind attention: the side stream
+ * copies the reassigned requests' blocks layer after layer, ahead of `stream`
+ * (the copied entries were committed before the round); `stream` waits for a
+ * layer's copy event (the KVReady condition of Eq. (F.3)), appends the new
+ * tokens of every request and attends.  The first layer, which has nothing
+ * else to hide its copy behind, appends and attends its resident requests
+ * before that wait and the reassigned ones after it.  Acceptance follows the
+ * last layer.  With num_slabs < num_layers the copy of layer l also waits for
+ * the attention of layer l - num_slabs.  Needs a plan for this batch.  Returns
+ * after enqueue; `stream` carries the completion.
  *
  * fuse_gather = 1 selects the gather-through variant (an extension beyond the
  * side-stream design; same pool bytes and outputs): there is no copy kernel and

@@ -577,28 +577,37 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
     }
     for (int l = 0; l < L; ++l) {
         uint16_t* slab = slab_ptr(ctx, a->kv_pool, l);
-        if (hook) {
-            NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_in[l], 0));
-            if (overlap) NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_in[l], 0));
-        }
+        if (hook) NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_in[l], 0));
         if (overlap) {
-            // side stream: copy + append of the reassigned requests of layer l
+            // Side stream: the copy of layer l's blocks.  It needs nothing this round computes (the copied entries
+            // were committed before the round), so it runs ahead of the main stream -- as many layers as there are
+            // spare slabs -- and the copy of layer l + 1 is under way while layer l attends: Run || Prepare, layer by
+            // layer.  The new tokens' rows, which a model only has once it reaches the layer, are appended on the
+            // main stream, for every request, right before the layer's attention.
             if (l >= S) NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_attn[l - S], 0));
             NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, a->mig_src, a->mig_dst, ctx->d_status, ctx->side));
-            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
-                                        k_new + l * kv_layer, v_new + l * kv_layer, a->is_migrated, 2, ctx->d_status, ctx->side));
             NSD_CUDA(ctx, cudaEventRecord(ctx->ev_prep[l], ctx->side));
-            ctx->launches += 2;
-            // main stream: resident requests, then the reassigned ones once their state is ready
-            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
-                                        k_new + l * kv_layer, v_new + l * kv_layer, a->is_migrated, 1, ctx->d_status, st));
             ctx->launches++;
-            nsd_status s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
-                                        a->kv_indptr, a->kv_indices, l, 1, st);
-            if (s != NSD_OK) return s;
-            NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_prep[l], 0));
-            s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
-                             a->kv_indptr, a->kv_indices, l, 2, st);
+            nsd_status s;
+            if (l == 0) {
+                // nothing to hide the first copy behind but the first layer itself: its resident requests go first
+                NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, k_new, v_new,
+                                            a->is_migrated, 1, ctx->d_status, st));
+                s = attn_enqueue(ctx, a->kv_pool, q, o, nullptr, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, 0, 1, st);
+                if (s != NSD_OK) return s;
+                NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_prep[0], 0));
+                NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, k_new, v_new,
+                                            a->is_migrated, 2, ctx->d_status, st));
+                s = attn_enqueue(ctx, a->kv_pool, q, o, nullptr, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, 0, 2, st);
+                ctx->launches += 2;
+            } else {
+                NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_prep[l], 0));
+                NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
+                                            k_new + l * kv_layer, v_new + l * kv_layer, nullptr, 0, ctx->d_status, st));
+                s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
+                                 a->kv_indptr, a->kv_indices, l, 0, st);
+                ctx->launches++;
+            }
             if (s != NSD_OK) return s;
             if (l + S < L) NSD_CUDA(ctx, cudaEventRecord(ctx->ev_attn[l], st));
         } else if (fused) {

@@ -150,5 +150,6 @@ def test_gather_through_needs_a_matching_plan():
 
 def test_launch_count_matches_the_choreography():
     ctx = _run_round(MULTI, 5)
-    # per layer: gather + reassigned append + resident append + 2 attention launches; one acceptance
-    assert ctx.nsd_launch_count() == 5 * 5 + 1
+    # per layer: the copy (side stream), one append and one attention launch; the first layer appends and attends its
+    # resident and its reassigned requests separately (two launches more); one acceptance
+    assert ctx.nsd_launch_count() == 5 * 3 + 2 + 1
