@@ -47,6 +47,7 @@ struct nsd_ctx {
     std::vector<CUtensorMap> tmaps;
     std::vector<const void*> tmap_slab;
     int n_sms;
+    int logits_feed;           // acceptance from logits: 1 = rows through the shared-memory ring where aligned (default), 0 = direct loads
     int attn_path;             // 0 = mma.sync kernel fed by cp.async, 1 = tcgen05 kernel where it applies, 2 = mma.sync fed by TMA where faster (default)
     int64_t launches;
     char err[256];
@@ -224,6 +225,11 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
         // (cp.async otherwise).  NSD_ATTN_PATH=mma forces cp.async everywhere, =tcgen05 selects the tcgen05 engine.
         const char* path = getenv("NSD_ATTN_PATH");
         ctx->attn_path = !path ? 2 : (strcmp(path, "tcgen05") == 0 ? 1 : (strcmp(path, "mma") == 0 ? 0 : 2));
+    }
+    {
+        // NSD_LOGITS_FEED=direct keeps the logits rows on direct loads (the ring of bulk copies is the default).
+        const char* feed = getenv("NSD_LOGITS_FEED");
+        ctx->logits_feed = (feed && strcmp(feed, "direct") == 0) ? 0 : 1;
     }
     *out = ctx;
     return NSD_OK;
@@ -522,8 +528,8 @@ nsd_status nsd_spec_accept_logits(nsd_ctx* ctx, const void* logits, int32_t logi
     if (temperature > 0.f && (!q || !u_acc || !u_smp)) return NSD_ERR_INVALID_ARG;
     if ((new_ctx_len != nullptr) && !ctx_len) return NSD_ERR_INVALID_ARG;
     NSD_CUDA(ctx, launch_accept_logits(logits, logits_dtype, temperature, q, draft_tok, u_acc, u_smp, batch, gamma, vocab,
-                                       gamma_r, ctx_len, acc_len, out_tok, new_ctx_len, ctx->d_status,
-                                       static_cast<cudaStream_t>(stream)));
+                                       gamma_r, ctx_len, acc_len, out_tok, new_ctx_len, ctx->d_status, ctx->n_sms,
+                                       ctx->logits_feed, static_cast<cudaStream_t>(stream)));
     ctx->launches++;
     return NSD_OK;
 }

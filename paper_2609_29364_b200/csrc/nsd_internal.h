@@ -97,6 +97,7 @@ cudaError_t launch_accept_logits(const void* logits, int32_t logits_bf16, float 
                                  const int32_t* draft_tok, const float* u_acc, const float* u_smp, int32_t batch,
                                  int32_t gamma, int32_t vocab, const int32_t* gamma_r, const int32_t* ctx_len,
                                  int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
+                                 int32_t n_sms, int32_t feed /* 0 = direct loads, 1 = shared-memory ring where aligned */,
                                  cudaStream_t stream);
 
 }  // namespace nsd

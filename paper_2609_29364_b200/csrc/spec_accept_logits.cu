@@ -13,6 +13,13 @@
 // Exponentials are ex2.approx in fp32 with log2(e)/T folded into the argument; sums and
 // compares are fp64.  A decision can therefore differ from an all-fp64 evaluation only
 // within fp32 rounding of p at a decision or CDF boundary.
+//
+// Feed.  Where rows start on 4-value boundaries (vocab a multiple of 4) they do not travel through
+// registers one load at a time: every thread copies its own 16-byte pieces (8 for bf16) of the
+// next tiles with cp.async into a ring of 8 KiB tiles in shared memory and reads them back
+// itself, so a CTA keeps 32-96 KiB in flight with no barrier of any kind and no registers
+// held.  Each thread sees the same elements in the same order as with direct loads, so the two
+// feeds give identical results; other shapes use direct loads.
 #include <cuda_bf16.h>
 
 #include "nsd_internal.h"
@@ -23,7 +30,9 @@ namespace {
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kSeg = 128;                       // tokens per segment of the draw
+constexpr int kAhead = 32;                      // drafts per request whose scalars are fetched ahead
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kStatsSlack = 8.0f;             // log2 units a logit may exceed the running reference by
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
@@ -65,32 +74,37 @@ struct Shared {
     float red_m[kWarps];
     double red_s[kWarps];
     int red_i[kWarps];
-    float row_max;        // M of the current row
+    float row_max;        // M of the current row: a reference within kStatsSlack (log2 units) of its maximum
     double row_sum;       // S = sum_k 2^((z_k - M) * c)
     int row_argmax;
     int n;                // accepted length once decided, else -1
     int found_seg;
     int token;
     double total;
+    int dx[kAhead];       // draft tokens, their uniforms and their draft probabilities, fetched ahead of the sweeps
+    float du[kAhead];
+    float dq[kAhead];
 };
 
-// Block-wide max and sum of exponentials of one row: every thread keeps a running (m, s) pair.
-template <typename T>
-__device__ void row_stats(const T* row, int vocab, bool vec_ok, float c, Shared& sh) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    float m = -INFINITY, s = 0.f;
-    const int n4 = (vocab + 3) / 4;
-#pragma unroll 4
-    for (int k4 = tid; k4 < n4; k4 += kThreads) {
-        const float4 z = load4(row, k4 * 4, vocab, vec_ok);
-        const float zm = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
-        if (zm > m) {
-            s *= ex2_approx((m - zm) * c);          // m = -inf: s is 0 and stays 0
-            m = zm;
-        }
-        if (m > -INFINITY)
-            s += ex2_approx((z.x - m) * c) + ex2_approx((z.y - m) * c) + ex2_approx((z.z - m) * c) + ex2_approx((z.w - m) * c);
+// Online update of one thread's running (reference, sum of exponentials relative to it) with four more logits.
+// The reference m is raised only when a logit exceeds it by more than `slack` (= kStatsSlack / c, i.e. when an
+// exponential would exceed 2^kStatsSlack): after the first tiles of a row that is rare, whereas an exact running
+// maximum changes in some lane of a warp on almost every iteration and makes the whole warp take the rescaling path.
+// Any reference gives the same softmax; the sums stay below 2^kStatsSlack * vocab, far inside fp32.
+__device__ __forceinline__ void stats_add4(const float4 z, float c, float slack, float& m, float& s) {
+    const float zm = fmaxf(fmaxf(z.x, z.y), fmaxf(z.z, z.w));
+    if (zm > m + slack) {
+        s *= ex2_approx((m - zm) * c);          // m = -inf: s is 0 and stays 0
+        m = zm;
     }
+    if (m > -INFINITY)
+        s += ex2_approx((z.x - m) * c) + ex2_approx((z.y - m) * c) + ex2_approx((z.z - m) * c) + ex2_approx((z.w - m) * c);
+}
+
+// Merges the threads' (m, s) pairs into the row's reference (the largest of the threads') and its sum
+// (sh.row_max, sh.row_sum).
+__device__ void stats_finish(float m, float s, float c, Shared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float wm = m;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
@@ -116,25 +130,33 @@ __device__ void row_stats(const T* row, int vocab, bool vec_ok, float c, Shared&
     __syncthreads();
 }
 
-// Block-wide argmax of one row: largest value, smallest index among equals, NaN never wins.
+// Block-wide max and sum of exponentials of one row, direct loads: every thread keeps a running (m, s) pair.
 template <typename T>
-__device__ void row_argmax(const T* row, int vocab, bool vec_ok, Shared& sh) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    float bv = -INFINITY;
-    int bi = -1;
+__device__ void row_stats(const T* row, int vocab, bool vec_ok, float c, Shared& sh) {
+    float m = -INFINITY, s = 0.f;
     const int n4 = (vocab + 3) / 4;
-    for (int k4 = tid; k4 < n4; k4 += kThreads) {
-        const float4 z = load4(row, k4 * 4, vocab, vec_ok);
-        const float v[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll 4
+    const float slack = kStatsSlack / c;
+    for (int k4 = threadIdx.x; k4 < n4; k4 += kThreads) stats_add4(load4(row, k4 * 4, vocab, vec_ok), c, slack, m, s);
+    stats_finish(m, s, c, sh);
+}
+
+// Running argmax of one thread: largest value, smallest index among equals, NaN never wins.
+__device__ __forceinline__ void argmax_add4(const float4 z, int k0, int vocab, float& bv, int& bi) {
+    const float v[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int k = k4 * 4 + j;
-            if (k < vocab && (v[j] > bv || (bi < 0 && v[j] == v[j]))) {      // strictly greater, or the first non-NaN
-                bv = v[j];
-                bi = k;
-            }
+    for (int j = 0; j < 4; ++j) {
+        const int k = k0 + j;
+        if (k < vocab && (v[j] > bv || (bi < 0 && v[j] == v[j]))) {      // strictly greater, or the first non-NaN
+            bv = v[j];
+            bi = k;
         }
     }
+}
+
+// Merges the threads' candidates into the row's argmax (sh.row_argmax).
+__device__ void argmax_finish(float bv, int bi, Shared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     auto better = [](float v1, int i1, float v2, int i2) {   // is (v1, i1) ahead of (v2, i2)?
         if (i1 < 0) return false;
         if (i2 < 0) return true;
@@ -165,7 +187,18 @@ __device__ void row_argmax(const T* row, int vocab, bool vec_ok, Shared& sh) {
     __syncthreads();
 }
 
+// Block-wide argmax of one row, direct loads.
+template <typename T>
+__device__ void row_argmax(const T* row, int vocab, bool vec_ok, Shared& sh) {
+    float bv = -INFINITY;
+    int bi = -1;
+    const int n4 = (vocab + 3) / 4;
+    for (int k4 = threadIdx.x; k4 < n4; k4 += kThreads) argmax_add4(load4(row, k4 * 4, vocab, vec_ok), k4 * 4, vocab, bv, bi);
+    argmax_finish(bv, bi, sh);
+}
+
 }  // namespace
 }  // namespace nsd
 
+#include "spec_accept_logits_ring.inc"
 #include "spec_accept_logits_kernel.inc"

@@ -137,6 +137,35 @@ def test_qwen3_vocab_bf16_logits():
     assert rep["len_exact"] >= B - 1
 
 
+@pytest.mark.parametrize("V,dtype,T", [(4104, 0, 0.8), (20488, 0, 1.0), (8200, 1, 1.0), (12296, 1, 0.0), (2052, 0, 0.0)])
+def test_ring_and_direct_feeds_agree_bit_for_bit(V, dtype, T, monkeypatch):
+    """Rows whose starts are 16-byte aligned travel through the shared-memory ring of bulk copies; NSD_LOGITS_FEED=direct
+    keeps them on direct loads.  Every thread sees the same elements in the same order, so nothing may differ.  The
+    vocabularies span several 8 KiB tiles with a ragged last one, both for the row sweep and for the draw."""
+    rng = np.random.default_rng(V)
+    B, g = 200, 5                                                      # more CTAs than SMs: the 8-slot ring
+    z, q, tok, ua, us = _inputs(rng, B, g, V, T if T > 0 else 1.0)
+    z[:, :, 5] = 0.25 * np.round(4 * z[:, :, 9])                       # some exact ties for the argmax
+    if dtype == 1:
+        z = W.bf16_to_f32(W.f32_to_bf16(z))
+    if T == 0:                                                         # greedy drafts: the argmax, a quarter of them wrong
+        tok = np.argmax(z[:, :g], axis=-1).astype(np.int32)
+        wrong = rng.random((B, g)) < 0.25
+        tok[wrong] = (tok[wrong] + 3) % V
+    res = {}
+    for feed in ("ring", "direct"):
+        monkeypatch.setenv("NSD_LOGITS_FEED", feed)
+        res[feed] = _gpu(z, dtype, T, q, tok, ua, us) if T > 0 else _gpu(z, dtype, 0.0, None, tok, None, None)
+    assert np.array_equal(res["ring"][0], res["direct"][0]) and np.array_equal(res["ring"][1], res["direct"][1])
+    acc_r, out_r, _ = oracle.spec_accept_logits(z, T, q, tok, ua, us) if T > 0 else oracle.spec_accept_logits(z, 0.0, None, tok, None, None)
+    if T > 0:
+        rep = _compare_sampled(z, T, q, tok, ua, us, res["ring"][0], res["ring"][1], acc_r, out_r)
+        assert rep["len_exact"] >= B - 1 and rep["tok_exact"] >= B - 4
+    else:
+        assert np.array_equal(res["ring"][0], acc_r) and np.array_equal(res["ring"][1], out_r)
+    assert len(set(acc_r.tolist())) >= 3
+
+
 def test_bad_arguments():
     import paper_2609_29364_b200 as nsd
 
