@@ -111,7 +111,12 @@ size_t nsd_kv_pool_bytes(const nsd_config* cfg);
 /* Builds a context on caller-provided DEVICE memory `d_workspace` (256-byte
  * aligned, at least nsd_workspace_bytes(cfg), zero-filled by this call on the
  * legacy default stream, which is synchronised before return).  The device
- * current at this call owns the context. */
+ * current at this call owns the context.
+ * Two environment variables, read here, select alternative kernels that compute
+ * the same results (for comparison runs; unset = the defaults):
+ *   NSD_ATTN_PATH    "mma" = attention tiles by cp.async for every shape,
+ *                    "tcgen05" = the tcgen05 attention engine where it applies
+ *   NSD_LOGITS_FEED  "direct" = nsd_spec_accept_logits reads rows with direct loads */
 nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace_bytes, nsd_ctx** out);
 nsd_status nsd_destroy(nsd_ctx* ctx);
 

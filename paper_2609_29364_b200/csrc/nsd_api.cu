@@ -455,10 +455,6 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
     a.counters = ctx->d_counters;
     a.status = ctx->d_status;
     a.m_rows = (ctx->cfg.num_q_heads / ctx->cfg.num_kv_heads) * (gamma + 1);
-    {
-        static const int stages = getenv("NSD_ATTN_STAGES") ? atoi(getenv("NSD_ATTN_STAGES")) : 0;
-        a.tune_stages = stages;
-    }
     if (subset == 0) { a.items = ctx->d_items_all; a.n_items = ctx->n_all; }
     else if (subset == 1) { a.items = ctx->d_items_split; a.n_items = ctx->n_res; }
     else { a.items = ctx->d_items_split + ctx->n_res; a.n_items = ctx->n_mig_items; }

@@ -58,7 +58,6 @@ struct AttnLaunch {
     int32_t* counters;           // [max_batch][Hkv], zero between launches
     int32_t* status;
     int32_t m_rows;              // (Hq/Hkv) * (gamma+1)
-    int32_t tune_stages;         // experiment knob: 0 = default pipeline depth
     int32_t tmap_valid;          // tmap describes pool_slab
     int32_t tma_feed;            // mma.sync kernel: fetch K/V tiles with tensor copies where the shape allows
     CUtensorMap tmap;

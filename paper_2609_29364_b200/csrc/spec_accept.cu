@@ -247,7 +247,6 @@ spec_accept_split_kernel(const float* __restrict__ p, const float* __restrict__ 
 
     const int r = blockIdx.x / split, part = blockIdx.x - r * split;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int n_warps = kAcceptThreads / 32;
     const int n_seg = (vocab + kSeg - 1) / kSeg;
     const float* p_req = p + (int64_t)r * (gamma + 1) * vocab;
     const float* q_req = q + (int64_t)r * gamma * vocab;

@@ -135,8 +135,8 @@ template <typename T>
 __device__ void row_stats(const T* row, int vocab, bool vec_ok, float c, Shared& sh) {
     float m = -INFINITY, s = 0.f;
     const int n4 = (vocab + 3) / 4;
-#pragma unroll 4
     const float slack = kStatsSlack / c;
+#pragma unroll 4
     for (int k4 = threadIdx.x; k4 < n4; k4 += kThreads) stats_add4(load4(row, k4 * 4, vocab, vec_ok), c, slack, m, s);
     stats_finish(m, s, c, sh);
 }

@@ -665,7 +665,6 @@ cudaError_t attn_init() {
     if ((e = init_one<DD, WW, TT, KK, SS>()) != cudaSuccess) return e;
     NSD_ATTN_SHAPES(NSD_INIT, 64, kStagesD64)
     NSD_ATTN_SHAPES(NSD_INIT, 128, kStagesD128)
-    NSD_INIT(128, 1, 3, 16, 3) NSD_INIT(128, 1, 3, 32, 2) NSD_INIT(128, 1, 3, 32, 3)
 #define NSD_INIT_TMA(DD, WW, TT, KK, SS) \
     if ((e = init_one<DD, WW, TT, KK, SS, true>()) != cudaSuccess) return e;
     NSD_ATTN_SHAPES(NSD_INIT_TMA, 128, kStagesD128)
@@ -687,11 +686,6 @@ cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
         if (nw == WW && ntw == TT) return launch_one<DD, WW, TT, KK, SS, true>(a, stream);
         NSD_ATTN_SHAPES(NSD_TMA_CASE, 128, kStagesD128)
 #undef NSD_TMA_CASE
-    }
-    if (a.shape.D == 128 && nw == 1 && ntw == 3) {      // experiment knob: tile keys * 10 + ring depth
-        if (a.tune_stages == 163) return launch_one<128, 1, 3, 16, 3>(a, stream);
-        if (a.tune_stages == 322) return launch_one<128, 1, 3, 32, 2>(a, stream);
-        if (a.tune_stages == 323) return launch_one<128, 1, 3, 32, 3>(a, stream);
     }
 #define NSD_CASE(DD, WW, TT, KK, SS) \
     if (a.shape.D == DD && nw == WW && ntw == TT) return launch_one<DD, WW, TT, KK, SS>(a, stream);
@@ -827,6 +821,5 @@ extern "C" nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_bl
     a.counters = reinterpret_cast<int32_t*>(base + kStaticOffCounters);
     a.status = reinterpret_cast<int32_t*>(base + kStaticOffStatus);
     a.m_rows = rows;
-    a.tune_stages = 0;
     return launch_attn(a, st) == cudaSuccess ? NSD_OK : NSD_ERR_CUDA;
 }
