@@ -116,7 +116,10 @@ size_t nsd_kv_pool_bytes(const nsd_config* cfg);
  * the same results (for comparison runs; unset = the defaults):
  *   NSD_ATTN_PATH    "mma" = attention tiles by cp.async for every shape,
  *                    "tcgen05" = the tcgen05 attention engine where it applies
- *   NSD_LOGITS_FEED  "direct" = nsd_spec_accept_logits reads rows with direct loads */
+ *   NSD_LOGITS_FEED  "direct" = nsd_spec_accept_logits reads rows with direct loads
+ *   NSD_ROUND_SPLIT  "always" / "never" = whether the first layer of a round attends its
+ *                    resident requests while the reassigned ones are still being copied
+ *                    (default: only when the copy is long enough to be worth a second launch) */
 nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace_bytes, nsd_ctx** out);
 nsd_status nsd_destroy(nsd_ctx* ctx);
 

@@ -47,6 +47,7 @@ struct nsd_ctx {
     std::vector<CUtensorMap> tmaps;
     std::vector<const void*> tmap_slab;
     int n_sms;
+    int round_split;           // first layer of a round with reassigned requests: 0 = by size, 1 = always attend resident and reassigned requests separately, 2 = never
     int logits_feed;           // acceptance from logits: 1 = rows through the shared-memory ring where aligned (default), 0 = direct loads
     int attn_path;             // 0 = mma.sync kernel fed by cp.async, 1 = tcgen05 kernel where it applies, 2 = mma.sync fed by TMA where faster (default)
     int64_t launches;
@@ -225,6 +226,11 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
         // (cp.async otherwise).  NSD_ATTN_PATH=mma forces cp.async everywhere, =tcgen05 selects the tcgen05 engine.
         const char* path = getenv("NSD_ATTN_PATH");
         ctx->attn_path = !path ? 2 : (strcmp(path, "tcgen05") == 0 ? 1 : (strcmp(path, "mma") == 0 ? 0 : 2));
+    }
+    {
+        // NSD_ROUND_SPLIT=always / never overrides the size rule for the first layer of a round (see round_impl).
+        const char* split = getenv("NSD_ROUND_SPLIT");
+        ctx->round_split = !split ? 0 : (strcmp(split, "always") == 0 ? 1 : (strcmp(split, "never") == 0 ? 2 : 0));
     }
     {
         // NSD_LOGITS_FEED=direct keeps the logits rows on direct loads (the ring of bulk copies is the default).
@@ -573,6 +579,12 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
     if (a->fuse_gather && n_pairs != ctx->plan_src_blocks) return NSD_ERR_INVALID_ARG;   // the plan walks the same list
     const bool fused = a->fuse_gather && n_pairs > 0;
     const bool overlap = n_pairs > 0 && !fused;
+    // The first layer has nothing to hide its copy behind but itself: its resident requests can be appended and
+    // attended while the copy runs, the reassigned ones after it.  That costs a second, partial attention launch
+    // (tens of microseconds of ramp and tail), so it only pays when the copy is longer than that: from about
+    // 60 us of copying (384 MiB read + written) on.  Below, the layer simply waits for its copy.
+    const int64_t copy_bytes = n_pairs * ctx->shape.block_elems() * 2 * (int64_t)sizeof(uint16_t);
+    const bool split_first = ctx->round_split == 1 || (ctx->round_split == 0 && copy_bytes >= (384LL << 20));
     if (overlap) {
         NSD_CUDA(ctx, cudaEventRecord(ctx->ev_start, st));
         NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_start, 0));
@@ -591,7 +603,7 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
             NSD_CUDA(ctx, cudaEventRecord(ctx->ev_prep[l], ctx->side));
             ctx->launches++;
             nsd_status s;
-            if (l == 0) {
+            if (l == 0 && split_first) {
                 // nothing to hide the first copy behind but the first layer itself: its resident requests go first
                 NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, k_new, v_new,
                                             a->is_migrated, 1, ctx->d_status, st));

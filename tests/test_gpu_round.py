@@ -25,6 +25,7 @@ def _oracle_round(cfg, meta, pool0, k_new, v_new, q, acc_in):
 
 
 def _run_round(cfg, slabs, host_variant=False, repeat=1, fuse=False):
+    """The context reads NSD_ROUND_SPLIT when it is made: the tests below set it to cover both first-layer orders."""
     meta = W.make_batch_meta(cfg)
     pool0 = np.stack([W.pool_layer(cfg, meta, s) for s in range(slabs)])
     k_new, v_new = stack_layers(cfg, meta, "kv")
@@ -99,18 +100,26 @@ def test_tiny_config_round():
     _run_round(W.CONFIGS["tiny"], 1)
 
 
+@pytest.mark.parametrize("split", ["always", "never"])
 @pytest.mark.parametrize("cfg,slabs", [(MULTI, 5), (MULTI, 2), (NOMIG, 2), (ALLMIG, 1), (ALLMIG, 3)],
                          ids=["multi", "multi_alias2", "nomig", "allmig_alias1", "allmig"])
-def test_multi_layer_round(cfg, slabs):
+def test_multi_layer_round(cfg, slabs, split, monkeypatch):
+    """Both orders of the first layer: resident requests attended while the copy runs and the reassigned ones after it
+    (what large copies get), or the whole layer after its copy (small copies)."""
+    monkeypatch.setenv("NSD_ROUND_SPLIT", split)
     _run_round(cfg, slabs)
 
 
-def test_round_twice_gives_the_same_state():
+@pytest.mark.parametrize("split", ["always", "never"])
+def test_round_twice_gives_the_same_state(split, monkeypatch):
     """The round is idempotent on its inputs (what the benchmark relies on)."""
+    monkeypatch.setenv("NSD_ROUND_SPLIT", split)
     _run_round(MULTI, 2, repeat=3)
 
 
-def test_host_buffer_round():
+@pytest.mark.parametrize("split", ["always", "never"])
+def test_host_buffer_round(split, monkeypatch):
+    monkeypatch.setenv("NSD_ROUND_SPLIT", split)
     _run_round(MULTI, 2, host_variant=True)
     _run_round(W.CONFIGS["tiny"], 1, host_variant=True, repeat=2)
 
@@ -148,8 +157,9 @@ def test_gather_through_needs_a_matching_plan():
     assert e.value.code == 1 and ctx.nsd_launch_count() == 0
 
 
-def test_launch_count_matches_the_choreography():
-    ctx = _run_round(MULTI, 5)
-    # per layer: the copy (side stream), one append and one attention launch; the first layer appends and attends its
-    # resident and its reassigned requests separately (two launches more); one acceptance
-    assert ctx.nsd_launch_count() == 5 * 3 + 2 + 1
+def test_launch_count_matches_the_choreography(monkeypatch):
+    # per layer: the copy (side stream), one append and one attention launch; one acceptance
+    assert _run_round(MULTI, 5).nsd_launch_count() == 5 * 3 + 1          # a small copy: the first layer waits for it
+    monkeypatch.setenv("NSD_ROUND_SPLIT", "always")
+    # the first layer appends and attends its resident and its reassigned requests separately: two launches more
+    assert _run_round(MULTI, 5).nsd_launch_count() == 5 * 3 + 2 + 1
