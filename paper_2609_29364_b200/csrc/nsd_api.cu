@@ -296,6 +296,17 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
         int64_t want = (total_blocks * Hkv + target_items - 1) / target_items;
         want = std::min<int64_t>(std::max<int64_t>(want, 16), 256);
         cb = (int)((want + 1) & ~1LL);
+        // Cutting each request into equal chunks of at most cb blocks rounds the item count up; where one wave is
+        // within reach (batch x kv heads fits the slots) lengthen the chunks until the items really fit it: a second
+        // wave of a few left-over CTAs costs far more than slightly longer chunks (batch 64: 1.13 waves before).
+        if ((int64_t)batch * Hkv <= target_items) {
+            auto n_items = [&](int c) {
+                int64_t n = 0;
+                for (int r = 0; r < batch; ++r) n += (nblk[r] + c - 1) / c;
+                return n;
+            };
+            while (cb < 256 && n_items(cb) * Hkv > target_items) cb += 2;
+        }
     }
     auto count_slots = [&](int c) {
         int64_t slots = 0;
