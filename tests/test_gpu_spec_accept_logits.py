@@ -137,13 +137,15 @@ def test_qwen3_vocab_bf16_logits():
     assert rep["len_exact"] >= B - 1
 
 
+@pytest.mark.parametrize("B", [200, 320], ids=["deep_ring", "four_per_sm"])
 @pytest.mark.parametrize("V,dtype,T", [(4104, 0, 0.8), (20488, 0, 1.0), (8200, 1, 1.0), (12296, 1, 0.0), (2052, 0, 0.0)])
-def test_ring_and_direct_feeds_agree_bit_for_bit(V, dtype, T, monkeypatch):
+def test_ring_and_direct_feeds_agree_bit_for_bit(V, dtype, T, B, monkeypatch):
     """Rows whose starts are 16-byte aligned travel through the shared-memory ring of bulk copies; NSD_LOGITS_FEED=direct
     keeps them on direct loads.  Every thread sees the same elements in the same order, so nothing may differ.  The
     vocabularies span several 8 KiB tiles with a ragged last one, both for the row sweep and for the draw."""
-    rng = np.random.default_rng(V)
-    B, g = 200, 5                                                      # more CTAs than SMs: the 8-slot ring
+    # batch 200: CTAs have an SM (nearly) to themselves and get the 12-tile ring; batch 320: four CTAs per SM, 4 tiles
+    rng = np.random.default_rng(V + B)
+    g = 5
     z, q, tok, ua, us = _inputs(rng, B, g, V, T if T > 0 else 1.0)
     z[:, :, 5] = 0.25 * np.round(4 * z[:, :, 9])                       # some exact ties for the argmax
     if dtype == 1:
