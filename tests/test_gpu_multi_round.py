@@ -1,6 +1,6 @@
 """Two consecutive verification rounds on one batch, chained the way a worker would chain them:
-round 1 (with reassigned requests) -> suffix commit to the export copy -> context lengths rolled forward
-by the accepted lengths -> round 2 appends over the rejected drafts.  Checked against the oracle run of
+the first verification round (with reassigned requests) -> suffix commit to the export copy -> context lengths rolled forward
+by the accepted lengths -> the second verification round appends over the rejected drafts.  Checked against the oracle run of
 the same sequence."""
 from dataclasses import replace
 
