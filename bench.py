@@ -465,7 +465,18 @@ def run_ours(args):
     ms_accept_logits = timed(accept_logits_only, max(5, args.steps), 2)
     acc2_h = acc2.cpu().numpy()
     bytes_accept_logits = int((acc2_h + 1).sum()) * cfg.vocab * 4 + int((acc2_h < cfg.gamma).sum()) * cfg.vocab * 4
+    # the same from bf16 logits (what a bf16 model head writes): half the bytes per swept row, its own decisions
+    logits16 = logits.to(torch.bfloat16).view(torch.int16)
     del logits
+
+    def accept_logits16_only():
+        ctx.nsd_spec_accept_logits(logits16, 1, 1.0, d["q_draft"], d["draft_tok"], d["u_acc"], d["u_smp"], B, cfg.gamma, cfg.vocab,
+                                   None, d["ctx_len"], acc2, out2, None, stream=stream)
+
+    ms_accept_logits16 = timed(accept_logits16_only, max(5, args.steps), 2)
+    acc3_h = acc2.cpu().numpy()
+    bytes_accept_logits16 = int((acc3_h + 1).sum()) * cfg.vocab * 2 + int((acc3_h < cfg.gamma).sum()) * cfg.vocab * 4
+    del logits16
     nomig = ctx.round_args(**{**d, "n_mig_blocks": 0, "mig_src": None, "mig_dst": None, "is_migrated": None})
     ms_round_nomig = timed(lambda: ctx.nsd_verify_round(nomig, stream=stream), max(2, args.steps // 2), 1)
     exposed_ms = ms_round - ms_round_nomig
@@ -563,7 +574,9 @@ def run_ours(args):
                              "accept_GBs_alone": bytes_["accept"] / (ms_accept * 1e-3) / 1e9,
                              "accept_from_logits_alone": ms_accept_logits,
                              "accept_from_logits_GBs": bytes_accept_logits / (ms_accept_logits * 1e-3) / 1e9,
-                             "accept_from_logits_agrees_on": float((acc2_h == acc_len).mean())},
+                             "accept_from_logits_agrees_on": float((acc2_h == acc_len).mean()),
+                             "accept_from_bf16_logits_alone": ms_accept_logits16,
+                             "accept_from_bf16_logits_GBs": bytes_accept_logits16 / (ms_accept_logits16 * 1e-3) / 1e9},
             "gather_through_round": {
                 "what": "nsd_verify_round with fuse_gather=1: attention reads reassigned requests from their source blocks and "
                         "writes the destination blocks itself; no copy kernel, no side stream; same pool bytes and outputs",
