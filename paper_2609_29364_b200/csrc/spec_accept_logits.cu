@@ -14,9 +14,9 @@
 // compares are fp64.  A decision can therefore differ from an all-fp64 evaluation only
 // within fp32 rounding of p at a decision or CDF boundary.
 //
-// Feed.  Where rows start on 4-value boundaries (vocab a multiple of 4) they do not travel through
-// registers one load at a time: every thread copies its own 16-byte pieces (8 for bf16) of the
-// next tiles with cp.async into a ring of 8 KiB tiles in shared memory and reads them back
+// Feed.  Where rows start on 16-byte boundaries and hold whole 16-byte pieces (vocab a multiple of
+// 4 for fp32, of 8 for bf16) they do not travel through registers one load at a time: every
+// thread copies its own 16-byte pieces of the next tiles with cp.async into a ring of 8 KiB tiles in shared memory and reads them back
 // itself, so a CTA keeps 32-96 KiB in flight with no barrier of any kind and no registers
 // held.  Each thread sees the same elements in the same order as with direct loads, so the two
 // feeds give identical results; other shapes use direct loads.
@@ -86,6 +86,46 @@ struct Shared {
     float dq[kAhead];
 };
 
+// Values one thread takes per iteration of a row sweep: one 16-byte piece (4 fp32 or 8 bf16 values).
+template <typename T>
+constexpr int kGroup = 16 / (int)sizeof(T);
+
+// Eight bf16 values held in four 32-bit words, as two groups of four floats.
+__device__ __forceinline__ void bf16x8_to_float(const uint4 raw, float4& lo, float4& hi) {
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x), b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+    const __nv_bfloat162 c = *reinterpret_cast<const __nv_bfloat162*>(&raw.z), d = *reinterpret_cast<const __nv_bfloat162*>(&raw.w);
+    lo = make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
+    hi = make_float4(__low2float(c), __high2float(c), __low2float(d), __high2float(d));
+}
+
+// Sweep of one row with direct loads: thread tid takes the groups tid, tid + 512, ... of kGroup<T> consecutive values
+// and hands them to add4(four values, index of the first), four at a time in index order.  (The shared-memory ring
+// walks the same elements in the same order.)
+template <typename T, class Add4>
+__device__ __forceinline__ void direct_sweep(const T* row, int vocab, bool vec_ok, Add4 add4) {
+    if constexpr (sizeof(T) == 4) {
+        const int n4 = (vocab + 3) / 4;
+#pragma unroll 4
+        for (int k4 = threadIdx.x; k4 < n4; k4 += kThreads) add4(load4(row, k4 * 4, vocab, vec_ok), k4 * 4);
+    } else {
+        const bool vec16_ok = (vocab % 8 == 0) && (reinterpret_cast<uintptr_t>(row) % 16 == 0);
+        const int n8 = (vocab + 7) / 8;
+#pragma unroll 2
+        for (int k8 = threadIdx.x; k8 < n8; k8 += kThreads) {
+            const int k0 = k8 * 8;
+            if (vec16_ok) {
+                float4 lo, hi;
+                bf16x8_to_float(__ldg(reinterpret_cast<const uint4*>(row + k0)), lo, hi);
+                add4(lo, k0);
+                add4(hi, k0 + 4);
+            } else {
+                add4(load4(row, k0, vocab, vec_ok), k0);
+                if (k0 + 4 < vocab) add4(load4(row, k0 + 4, vocab, vec_ok), k0 + 4);
+            }
+        }
+    }
+}
+
 // Online update of one thread's running (reference, sum of exponentials relative to it) with four more logits.
 // The reference m is raised only when a logit exceeds it by more than `slack` (= kStatsSlack / c, i.e. when an
 // exponential would exceed 2^kStatsSlack): after the first tiles of a row that is rare, whereas an exact running
@@ -130,14 +170,12 @@ __device__ void stats_finish(float m, float s, float c, Shared& sh) {
     __syncthreads();
 }
 
-// Block-wide max and sum of exponentials of one row, direct loads: every thread keeps a running (m, s) pair.
+// Block-wide reference and sum of exponentials of one row, direct loads: every thread keeps a running (m, s) pair.
 template <typename T>
 __device__ void row_stats(const T* row, int vocab, bool vec_ok, float c, Shared& sh) {
     float m = -INFINITY, s = 0.f;
-    const int n4 = (vocab + 3) / 4;
     const float slack = kStatsSlack / c;
-#pragma unroll 4
-    for (int k4 = threadIdx.x; k4 < n4; k4 += kThreads) stats_add4(load4(row, k4 * 4, vocab, vec_ok), c, slack, m, s);
+    direct_sweep(row, vocab, vec_ok, [&](const float4 z, int) { stats_add4(z, c, slack, m, s); });
     stats_finish(m, s, c, sh);
 }
 
@@ -192,8 +230,7 @@ template <typename T>
 __device__ void row_argmax(const T* row, int vocab, bool vec_ok, Shared& sh) {
     float bv = -INFINITY;
     int bi = -1;
-    const int n4 = (vocab + 3) / 4;
-    for (int k4 = threadIdx.x; k4 < n4; k4 += kThreads) argmax_add4(load4(row, k4 * 4, vocab, vec_ok), k4 * 4, vocab, bv, bi);
+    direct_sweep(row, vocab, vec_ok, [&](const float4 z, int k0) { argmax_add4(z, k0, vocab, bv, bi); });
     argmax_finish(bv, bi, sh);
 }
 
