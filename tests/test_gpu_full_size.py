@@ -136,3 +136,34 @@ def test_long_b128():
     if not FULL:
         cfg = W.RoundConfig(**{**cfg.__dict__, "batch": 12})
     _full_round_check(cfg, slabs=2, layers_to_check=[1, 34], slabs_to_check=[0])
+
+
+def test_knee_b512_acceptance_from_logits_full_size():
+    """nsd_spec_accept_logits in the launch configuration the benchmark times (batch 512, the Qwen3 vocabulary, fp32
+    logits = log p of the configuration's acceptance inputs, T = 1: one wave of 512 CTAs, four per SM, the four-tile
+    ring), every request launched, a sample of them checked against the logits oracle one by one; and the same decisions
+    as nsd_spec_accept on the probabilities themselves wherever no test sits on a boundary."""
+    cfg = W.CONFIGS["knee_b512"]
+    meta = W.make_batch_meta(cfg)
+    B, g, V = cfg.batch, cfg.gamma, cfg.vocab
+    p, qd, tok, ua, us = W.accept_inputs(cfg)
+    with np.errstate(divide="ignore"):
+        z = np.log(p.astype(np.float64)).astype(np.float32)           # what both sides see
+    ctx = make_context(cfg, meta, num_slabs=1)
+    acc = torch.full((B,), -7, dtype=torch.int32, device="cuda:0")
+    out = torch.full((B, g + 1), -7, dtype=torch.int32, device="cuda:0")
+    ctx.nsd_spec_accept_logits(dev(z), 0, 1.0, dev(qd), dev(tok), dev(ua), dev(us), B, g, V, None, None, acc, out, None)
+    rc, bad = ctx.nsd_get_status()
+    assert rc == 0, (rc, bad)
+    acc_g, out_g = acc.cpu().numpy(), out.cpu().numpy()
+
+    sel = np.sort(np.random.default_rng(cfg.seed).choice(B, size=48, replace=False))
+    acc_r, out_r, _ = oracle.spec_accept_logits(z[sel], 1.0, qd[sel], tok[sel], ua[sel], us[sel])
+    pz = np.exp(z[sel].astype(np.float64))
+    pz /= pz.sum(axis=-1, keepdims=True)
+    rep = accept_compare(pz.astype(np.float32), qd[sel], tok[sel], ua[sel], us[sel], acc_g[sel], out_g[sel], acc_r, out_r)
+    assert rep["len_exact"] >= len(sel) - 1, rep
+    print("acceptance from logits:", rep)
+    acc_p, _, _ = oracle.spec_accept(p, qd, tok, ua, us)
+    assert (acc_g == acc_p).mean() > 0.99
+    assert ((out_g >= -1) & (out_g < V)).all() and (acc_g >= 0).all() and (acc_g <= g).all()
