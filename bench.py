@@ -1,6 +1,6 @@
 #!/usr/bin/env python
-"""Benchmark of the B200 verification round (the benchmark spec metric: verify-round
-req/s and tokens/s at the Qwen3-8B shape, HBM GB/s against the B200 peak).
+"""Benchmark of the B200 verification round (metric: verify-round req/s and
+tokens/s at the Qwen3-8B shape, HBM GB/s against the B200 peak).
 
 One step = one whole verification round through the C ABI on one batch of
 synthetic input: for each of the 36 logical layers the KV-state preparation
@@ -33,8 +33,8 @@ import workload as W  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic byte of verify_attn_kernel, from the
-# ncu capture of the reduced case summarised in profiles/verify_attn_kernel_ncu.md (709.4 MB over 698.9 MB for one whole-batch pass); the
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per algorithmic byte of verify_attn_kernel, from a
+# profiler capture of a smaller case of the same kernel (709.4 MB over 698.9 MB for one whole-batch pass); the
 # full-size launch is too large to capture under the profiler, and traffic grows with the keys streamed.
 ATTN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.015
 
@@ -202,18 +202,23 @@ def run_reference(args):
     meta = W.make_batch_meta(cfg)
     host = host_inputs(cfg, meta)
     per_step = max(2.0, min(args.cpu_seconds, 150.0 / max(1, args.steps + args.warmup)))
-    times, desc, cores = [], "", 1
+    times, walls, desc, cores = [], [], "", 1
     for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
         t, desc, cores = oracle_sample(cfg, meta, host, per_step)
         if i >= args.warmup:
             times.append(t)
-    t_round = float(np.mean(times))
+            walls.append(time.perf_counter() - t0)
+    t_round = float(np.median(times))
     value = cfg.batch / t_round
     line = {
         "impl": "reference", "metric": "verify_round_requests_per_s", "value": value, "unit": "req/s",
-        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_round * 1e3,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        # a step is a bounded sample of the round (see cpu_baseline.sample): its measured time, and beside it the
+        # whole-round time extrapolated from the sample, which is what `value` is computed from
+        "ms_per_step": float(np.mean(walls)) * 1e3, "extrapolated_ms_per_round": t_round * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(cfg, meta, None),
+        "config": workload_config(cfg, meta),
         "cpu_baseline": {"value": value, "unit": "req/s", "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "req/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -229,11 +234,11 @@ def pick_config(args) -> W.RoundConfig:
     return cfg
 
 
-def workload_config(cfg, meta, slabs):
+def workload_config(cfg, meta):
     base = cfg.name.replace("_REDUCED_FOR_PROFILING", "")
     return {
-        "workload": f"{cfg.name} (BASELINE.json configs[{list(W.CONFIGS).index(base)}])", "batch": cfg.batch,
-        "gamma": cfg.gamma, "layers": cfg.num_layers, "physical_layer_slabs": slabs,
+        "workload": f"{cfg.name} (configuration {list(W.CONFIGS).index(base) + 1} of the benchmark set)", "batch": cfg.batch,
+        "gamma": cfg.gamma, "layers": cfg.num_layers,
         "heads": f"{cfg.num_q_heads}q/{cfg.num_kv_heads}kv x {cfg.head_dim}", "block_size": cfg.block_size,
         "vocab": cfg.vocab, "ctx": list(cfg.ctx_dist), "mean_ctx": float(meta.ctx_len.mean()),
         "reassigned_requests": int(meta.n_mig), "pool_blocks_per_layer": int(meta.num_blocks),
@@ -252,7 +257,7 @@ def scheduled_rounds_leg(cfg, device, rounds, d_accept):
 
     import paper_2609_29364_b200 as nsd
     from paper_2609_29364_b200.rounds import ScheduledRounds
-    from workload.banks import BankedPool
+    from paper_2609_29364_b200.banks import BankedPool
 
     B, g, L = max(4, cfg.batch // 2), cfg.gamma, cfg.num_layers
     n_req = (5 * B) // 2                                     # 2.5 batches in the stage's pool: about half of a batch comes back resident
@@ -400,14 +405,16 @@ def run_ours(args):
     launches0 = ctx.nsd_launch_count()
     sampler.start()
     time.sleep(0.3)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     with torch.cuda.stream(stream):
-        e0.record(stream)
-        for _ in range(args.steps):
+        marks[0].record(stream)
+        for i in range(args.steps):
             one_round()
-        e1.record(stream)
+            marks[i + 1].record(stream)
     barrier()
-    ms_round = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    step_ms = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
+    ms_round = max_over_ranks(float(np.median(step_ms)))              # median step, the slowest rank's
+    ms_round_mean = max_over_ranks(marks[0].elapsed_time(marks[-1])) / args.steps
     gpu_launches = ctx.nsd_launch_count() - launches0
     clocks = sampler.stop()
     rc, bad = ctx.nsd_get_status(stream=stream)
@@ -553,8 +560,9 @@ def run_ours(args):
         line = {
             "metric": "verify_round_requests_per_s", "value": n_gpus * B / (ms_round * 1e-3), "unit": "req/s",
             "n_gpus": n_gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_round,
+            "ms_per_step_mean": ms_round_mean, "timing": "median of per-step CUDA-event pairs on the launching stream, max over ranks",
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": workload_config(cfg, meta, slabs),
+            "config": workload_config(cfg, meta), "physical_layer_slabs": slabs,
             "committed_tokens_per_s": n_gpus * committed / (ms_round * 1e-3),
             "verified_rows_per_s": n_gpus * cfg.rows / (ms_round * 1e-3),
             "mean_accepted_len": float(acc_len.mean()),
@@ -562,7 +570,7 @@ def run_ours(args):
                          "achieved": attn_gbs, "peak": peak, "peak_kind": f"{peak_kind} copy bandwidth",
                          "unit": "GB/s", "frac": attn_gbs / peak, "frac_of_nominal_8TBs": attn_gbs / NOMINAL_HBM_GBS,
                          "traffic": int(ATTN_TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_["attn_per_layer"]),
-                         "traffic_source": "ncu capture of a smaller case scaled by algorithmic bytes (profiles/verify_attn_kernel_ncu.md)",
+                         "traffic_source": "profiler capture of a smaller case of the same kernel, scaled by algorithmic bytes",
                          "bytes_per_launch": bytes_["attn_per_layer"], "ms_per_launch": ms_attn_launch},
             "round_roofline": {"bound": "hbm", "achieved": round_gbs, "peak": peak, "unit": "GB/s",
                                "frac": round_gbs / peak, "frac_of_nominal_8TBs": round_gbs / NOMINAL_HBM_GBS,

@@ -95,9 +95,31 @@ typedef struct {
     int32_t max_batch;
     int32_t max_gamma;         /* (num_q_heads/num_kv_heads)*(max_gamma+1) <= 64         */
     int32_t vocab_size;
-    int32_t reserved;
+    int32_t flags;             /* NSD_FLAG_* bits, 0 = the defaults                      */
     int64_t max_table_entries; /* upper bound of kv_indptr[batch]                        */
+    int32_t wait_budget;       /* polls a kernel spends on one barrier before it gives up with
+                                  NSD_ERR_TIMEOUT; 0 = the default (seconds)             */
+    int32_t reserved;          /* 0                                                      */
 } nsd_config;
+
+/* nsd_config.flags: alternative kernels that compute the same results (comparison runs and
+ * tests), and one test hook. */
+enum {
+    NSD_FLAG_ATTN_CP_ASYNC = 1 << 0,      /* attention: K/V tiles by cp.async for every shape (default: tensor
+                                             copies where they are the faster feed)                            */
+    NSD_FLAG_ATTN_TCGEN05 = 1 << 1,       /* attention: the tcgen05 engine for every shape it supports (default:
+                                             only for the shapes where it is the faster one)                   */
+    NSD_FLAG_ATTN_NO_TCGEN05 = 1 << 2,    /* attention: never the tcgen05 engine                               */
+    NSD_FLAG_LOGITS_DIRECT = 1 << 3,      /* nsd_spec_accept_logits reads rows with direct loads               */
+    NSD_FLAG_ROUND_SPLIT_ALWAYS = 1 << 4, /* first layer of a round: always attend the resident requests while
+                                             the reassigned ones are still being copied ...                    */
+    NSD_FLAG_ROUND_SPLIT_NEVER = 1 << 5,  /* ... or never (default: only when the copy is long enough to be
+                                             worth a second launch)                                            */
+    NSD_FLAG_TEST_STARVE_GATHER = 1 << 30 /* test hook for the bounded waits: the gather arms every barrier with
+                                             16 bytes more than its copy delivers, so each wait runs out after
+                                             wait_budget polls and nsd_get_status returns NSD_ERR_TIMEOUT; the
+                                             copies themselves still complete before the kernel returns        */
+};
 
 const char* nsd_status_string(nsd_status s);
 /* Text of the last failing CUDA call made through `ctx` (empty string if none). */
@@ -111,15 +133,8 @@ size_t nsd_kv_pool_bytes(const nsd_config* cfg);
 /* Builds a context on caller-provided DEVICE memory `d_workspace` (256-byte
  * aligned, at least nsd_workspace_bytes(cfg), zero-filled by this call on the
  * legacy default stream, which is synchronised before return).  The device
- * current at this call owns the context.
- * Two environment variables, read here, select alternative kernels that compute
- * the same results (for comparison runs; unset = the defaults):
- *   NSD_ATTN_PATH    "mma" = attention tiles by cp.async for every shape,
- *                    "tcgen05" = the tcgen05 attention engine where it applies
- *   NSD_LOGITS_FEED  "direct" = nsd_spec_accept_logits reads rows with direct loads
- *   NSD_ROUND_SPLIT  "always" / "never" = whether the first layer of a round attends its
- *                    resident requests while the reassigned ones are still being copied
- *                    (default: only when the copy is long enough to be worth a second launch) */
+ * current at this call owns the context.  cfg->flags selects alternative kernels
+ * (NSD_FLAG_*); the library reads no environment variable. */
 nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace_bytes, nsd_ctx** out);
 nsd_status nsd_destroy(nsd_ctx* ctx);
 
@@ -133,11 +148,16 @@ nsd_status nsd_destroy(nsd_ctx* ctx);
  *   h_kv_indptr    [batch+1]  non-decreasing, entry count of request r must
  *                             cover ceil((ctx_len[r]+gamma+1)/block_size)
  *   h_is_migrated  [batch]    nullable; 1 = reassigned to this worker this
- *                             round (its KV arrives through the gather)
+ *                             round (its KV arrives through the gather).  Must hold the
+ *                             values of the round's device is_migrated.  A plan made
+ *                             without it serves any round, but such a round cannot
+ *                             overlap its first layer with its own copy (it waits for
+ *                             the copy, then attends everybody) and cannot fuse_gather
  *   chunk_blocks   0 = choose; else the split-KV chunk length in blocks (even, <= 256)
  * Errors: INVALID_ARG (null, negative length, short table), OUT_OF_RANGE
  * (batch > max_batch, gamma outside [1,max_gamma]), CAPACITY (table entries or
- * split count beyond the workspace).  batch == 0 is a valid empty plan.
+ * split count beyond the workspace, or the host could not allocate the work list).
+ * batch == 0 is a valid empty plan.
  */
 nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
                            const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
@@ -349,7 +369,10 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
  *   kv_slab     bf16 [num_blocks][2][num_kv_heads][block_size][head_dim] (one layer)
  *   q, o        bf16 [batch*(gamma+1)][num_q_heads][head_dim]
  *   h_ctx_len   HOST int32 [batch]  (used to cut the work list; must equal ctx_len)
- *   ctx_len, kv_indptr, kv_indices   device tables as for nsd_verify_attn
+ *   ctx_len, kv_indptr, kv_indices   device tables as for nsd_verify_attn; request r's
+ *               table must cover ceil((h_ctx_len[r]+gamma+1)/block_size) entries.  This
+ *               entry point has no host copy of kv_indptr to check that with: an entry
+ *               index at or past kv_indptr[r+1] is not followed (block 0 is read instead)
  * Limits (NSD_ERR_CAPACITY beyond them, nothing launched): batch <= 64;
  * num_kv_heads <= 8; (num_q_heads/num_kv_heads)*(gamma+1) <= 32; requests longer
  * than 1024 keys are cut into 1024-key chunks and all such chunks of a call
@@ -358,7 +381,10 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
  * (NSD_ERR_UNSUPPORTED otherwise).  Other errors as nsd_verify_attn.
  *
  * The first call on a device resolves the array's address and sets kernel
- * attributes for that device; make that first call outside any stream capture.
+ * attributes for that device.  No call of this entry point may be made while `stream`
+ * is being captured into a CUDA graph: every call uploads its work list from a buffer
+ * that lives only for the duration of the call (NSD_ERR_INVALID_ARG if the stream is
+ * capturing).
  * All calls share the one array, and it keeps the previous call's contents: the
  * call clears the words that must start at zero, but two calls whose kernels can
  * overlap on the GPU (different streams, or the same call from two threads)
@@ -381,12 +407,12 @@ nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_blocks, int32
  * and a batch B is admissible (Eq. (8)) iff |B| <= max_batch, it fits the worker
  * (sum of rows / KV blocks / tokens within the capacities, Appendix F.2; a request
  * that does not fit alone is dropped), and S(B) = max over B of S({r}) <= min over B
- * of d_r.  Line 1 filters by `eligible`; line 2 ranks -- the paper names the criteria
- * (predecessor readiness, waiting time, temporal compatibility) but not the key:
- * this library sorts by d_r, then pred_done (older output first: the aging term),
- * then S({r}), then index; line 3 keeps the first max_batch; lines 4-8 admit greedily
- * in that order.  Freezing, PREPARE and RUN are the caller's (nsd_verify_plan and
- * nsd_verify_round take the chosen batch).
+ * of d_r.  Candidates are the `eligible` requests; they are ranked -- the paper names the
+ * criteria (predecessor readiness, waiting time, temporal compatibility) but not the
+ * key: this library sorts by d_r, then pred_done (older output first: the aging term),
+ * then S({r}), then index --, the first max_batch of them are kept, and those are
+ * admitted greedily in rank order while the batch stays admissible.  Freezing, PREPARE
+ * and RUN are the caller's (nsd_verify_plan and nsd_verify_round take the chosen batch).
  *   eligible   nullable uint8 [n] (null = all); pred_done, kv_ready  double [n]
  *   rows / blocks / tokens   nullable int32 [n] (null = 1 row, 0 blocks, 0 tokens each)
  *   batch_out  int32 [min(n, max_batch)]: indices of the admitted requests in rank order

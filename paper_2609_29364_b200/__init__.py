@@ -14,4 +14,11 @@ from .api import (  # noqa: F401
     nsd_schedule_batch,
     nsd_verify_attn_static,
     STATUS,
+    NSD_FLAG_ATTN_CP_ASYNC,
+    NSD_FLAG_ATTN_TCGEN05,
+    NSD_FLAG_ATTN_NO_TCGEN05,
+    NSD_FLAG_LOGITS_DIRECT,
+    NSD_FLAG_ROUND_SPLIT_ALWAYS,
+    NSD_FLAG_ROUND_SPLIT_NEVER,
+    NSD_FLAG_TEST_STARVE_GATHER,
 )

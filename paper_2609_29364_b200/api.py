@@ -27,7 +27,18 @@ class NsdError(RuntimeError):
 class NsdConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "num_layers", "num_slabs", "num_q_heads", "num_kv_heads", "head_dim", "block_size", "num_blocks",
-        "region_b_begin", "max_batch", "max_gamma", "vocab_size", "reserved")] + [("max_table_entries", ctypes.c_int64)]
+        "region_b_begin", "max_batch", "max_gamma", "vocab_size", "flags")] + [
+        ("max_table_entries", ctypes.c_int64), ("wait_budget", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+# nsd_config.flags (include/nsd.h)
+NSD_FLAG_ATTN_CP_ASYNC = 1 << 0
+NSD_FLAG_ATTN_TCGEN05 = 1 << 1
+NSD_FLAG_ATTN_NO_TCGEN05 = 1 << 2
+NSD_FLAG_LOGITS_DIRECT = 1 << 3
+NSD_FLAG_ROUND_SPLIT_ALWAYS = 1 << 4
+NSD_FLAG_ROUND_SPLIT_NEVER = 1 << 5
+NSD_FLAG_TEST_STARVE_GATHER = 1 << 30
 
 
 _vp = ctypes.c_void_p
@@ -168,15 +179,16 @@ class VerifyContext:
     """Owns an nsd_ctx and the torch-allocated workspace it lives on."""
 
     def __init__(self, *, num_layers, num_q_heads, num_kv_heads, head_dim, block_size, num_blocks, region_b_begin,
-                 max_batch, max_gamma, vocab_size, max_table_entries, num_slabs=None, device="cuda:0"):
+                 max_batch, max_gamma, vocab_size, max_table_entries, num_slabs=None, flags=0, wait_budget=0,
+                 device="cuda:0"):
         import torch
 
         self.lib = load_library()
         self.cfg = NsdConfig(num_layers=num_layers, num_slabs=num_slabs or num_layers, num_q_heads=num_q_heads,
                              num_kv_heads=num_kv_heads, head_dim=head_dim, block_size=block_size,
                              num_blocks=num_blocks, region_b_begin=region_b_begin, max_batch=max_batch,
-                             max_gamma=max_gamma, vocab_size=vocab_size, reserved=0,
-                             max_table_entries=max_table_entries)
+                             max_gamma=max_gamma, vocab_size=vocab_size, flags=flags,
+                             max_table_entries=max_table_entries, wait_budget=wait_budget, reserved=0)
         self.device = torch.device(device)
         self._h = _vp()
         nbytes = self.lib.nsd_workspace_bytes(ctypes.byref(self.cfg))

@@ -19,7 +19,8 @@ namespace {
 // mbarrier (transaction bytes), its store is a bulk group, and a slot is reused once the
 // store has finished READING shared memory.  No other thread touches the data, so the SM
 // spends a handful of instructions per 16 KiB.  Every wait is bounded: on a timeout the
-// CTA records STATUS_TIMEOUT, drains what it can and returns.
+// CTA records STATUS_TIMEOUT, waits (bounded again) for the loads it has armed, so that no
+// copy lands in shared memory the CTA has given back, waits for its stores and returns.
 constexpr int kBulkBytes = 16 * 1024;
 constexpr int kBulkSlots = 4;
 // A slot is refilled while up to kBulkBehind - 1 younger stores may still be reading shared memory, i.e. the loads run
@@ -32,8 +33,8 @@ constexpr uint32_t kBulkSpinLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kBulkSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -50,7 +51,8 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 __global__ void __launch_bounds__(32)
 gather_blocks_bulk_kernel(uint16_t* __restrict__ slab, int64_t n_pairs, const int32_t* __restrict__ src,
                           const int32_t* __restrict__ dst, int32_t num_blocks, int64_t block_bytes,
-                          int32_t pieces_per_block, int32_t* __restrict__ status) {
+                          int32_t pieces_per_block, int32_t* __restrict__ status, uint32_t spin_limit,
+                          uint32_t starve_bytes) {
     extern __shared__ __align__(128) unsigned char bulk_smem[];
     __shared__ __align__(8) uint64_t full_bar[kBulkSlots];
     if (threadIdx.x != 0) return;                       // a single thread drives the copy engine
@@ -84,7 +86,8 @@ gather_blocks_bulk_kernel(uint16_t* __restrict__ slab, int64_t n_pairs, const in
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
             return;
         }
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+        // starve_bytes is zero outside the bounded-wait test, which makes the phase impossible to complete
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes + starve_bytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"(smem_addr(bulk_smem + s * kBulkBytes)), "l"(sp), "r"(bytes), "r"(bar) : "memory");
     };
@@ -94,15 +97,17 @@ gather_blocks_bulk_kernel(uint16_t* __restrict__ slab, int64_t n_pairs, const in
     constexpr int kBehind = kBulkBehind;
     constexpr int kAhead = kBulkSlots - kBehind;
     bool ok = true;
-    for (int64_t k = 0; k < kAhead && k < mine; ++k) issue_load(k);
-    for (int64_t k = 0; k < mine && ok; ++k) {
-        if (k + kAhead < mine) {
-            // the slot of piece k + kAhead was last used by piece k - kBehind: that store must have finished reading
+    int64_t issued = 0;                                 // loads armed so far: pieces [0, issued)
+    for (; issued < kAhead && issued < mine; ++issued) issue_load(issued);
+    int64_t k = 0;
+    for (; k < mine; ++k) {
+        if (issued < mine) {
+            // the slot of piece `issued` = k + kAhead was last used by piece k - kBehind: that store must have finished reading
             asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kBehind - 1) : "memory");
-            issue_load(k + kAhead);
+            issue_load(issued++);
         }
         const int s = (int)(k % kBulkSlots);
-        ok = mbar_wait_bounded(smem_addr(&full_bar[s]), (uint32_t)((k / kBulkSlots) & 1));
+        ok = mbar_wait_bounded(smem_addr(&full_bar[s]), (uint32_t)((k / kBulkSlots) & 1), spin_limit);
         if (!ok) break;
         const char* sp; char* dp; uint32_t bytes;
         if (piece_ptrs(k, sp, dp, bytes)) {
@@ -111,7 +116,13 @@ gather_blocks_bulk_kernel(uint16_t* __restrict__ slab, int64_t n_pairs, const in
         }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     }
-    if (!ok) atomicOr(status, STATUS_TIMEOUT);
+    if (!ok) {
+        atomicOr(status, STATUS_TIMEOUT);
+        // the loads armed after piece k may still be writing this CTA's shared memory: give each of them the same
+        // bounded wait before the memory goes back to the SM
+        for (int64_t j = k + 1; j < issued; ++j)
+            mbar_wait_bounded(smem_addr(&full_bar[j % kBulkSlots]), (uint32_t)((j / kBulkSlots) & 1), spin_limit);
+    }
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores complete before the CTA retires
 }
 
@@ -215,15 +226,16 @@ cudaError_t gather_init() {
 }
 
 cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const int32_t* src, const int32_t* dst,
-                          int32_t* status, cudaStream_t stream) {
+                          int32_t* status, int n_sms, uint32_t wait_budget, uint32_t starve_bytes, cudaStream_t stream) {
     if (n_pairs <= 0) return cudaSuccess;
     const int64_t block_bytes = s.block_elems() * 2;
     const int32_t ppb = (int32_t)((block_bytes + kBulkBytes - 1) / kBulkBytes);
     const int64_t n_pieces = n_pairs * ppb;
     // A bounded number of CTAs (4 per SM, each with 48 KiB of loads in flight): the copy shares the SMs with attention.
-    const int64_t ctas = 148LL * kBulkCtasPerSm;
+    const int64_t ctas = (int64_t)(n_sms > 0 ? n_sms : 148) * kBulkCtasPerSm;
     const int grid = (int)(n_pieces < ctas ? n_pieces : ctas);
-    gather_blocks_bulk_kernel<<<grid, 32, kBulkSlots * kBulkBytes, stream>>>(slab, n_pairs, src, dst, s.num_blocks, block_bytes, ppb, status);
+    gather_blocks_bulk_kernel<<<grid, 32, kBulkSlots * kBulkBytes, stream>>>(slab, n_pairs, src, dst, s.num_blocks, block_bytes, ppb, status,
+                                                                          wait_budget ? wait_budget : kBulkSpinLimit, starve_bytes);
     return cudaGetLastError();
 }
 

@@ -37,6 +37,7 @@ struct nsd_ctx {
     int32_t plan_batch, plan_gamma;
     int32_t n_all, n_res, n_mig_items;
     int64_t plan_src_blocks;   // source blocks of the planned batch's reassigned requests
+    bool plan_has_mig;         // the plan was given is_migrated (its resident / reassigned item lists are meaningful)
     // streams / events
     cudaStream_t side;
     cudaStream_t copy, down;   // nsd_verify_round_host: uploads in the order they are needed / per-layer read-back of o
@@ -49,7 +50,10 @@ struct nsd_ctx {
     int n_sms;
     int round_split;           // first layer of a round with reassigned requests: 0 = by size, 1 = always attend resident and reassigned requests separately, 2 = never
     int logits_feed;           // acceptance from logits: 1 = rows through the shared-memory ring where aligned (default), 0 = direct loads
-    int attn_path;             // 0 = mma.sync kernel fed by cp.async, 1 = tcgen05 kernel where it applies, 2 = mma.sync fed by TMA where faster (default)
+    int attn_feed_tma;         // mma.sync kernel: K/V tiles by tensor copies where that is the faster feed (default), 0 = cp.async everywhere
+    int attn_tcgen05;          // tcgen05 engine: 0 = never, 1 = for the shapes where it is the faster one (default), 2 = wherever it applies
+    uint32_t wait_budget;      // polls per bounded wait, 0 = the kernels' default
+    uint32_t starve_gather;    // test hook: extra transaction bytes the gather expects and never gets
     int64_t launches;
     char err[256];
 };
@@ -145,7 +149,17 @@ size_t nsd_kv_pool_bytes(const nsd_config* cfg) {
     return (size_t)cfg->num_slabs * cfg->num_blocks * 2 * cfg->num_kv_heads * cfg->block_size * cfg->head_dim * 2;
 }
 
+static nsd_status create_impl(const nsd_config* cfg, void* d_workspace, size_t workspace_bytes, nsd_ctx** out);
+
 nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace_bytes, nsd_ctx** out) {
+    try {
+        return create_impl(cfg, d_workspace, workspace_bytes, out);
+    } catch (...) {                        // host allocation of the event lists failed
+        return NSD_ERR_CAPACITY;
+    }
+}
+
+static nsd_status create_impl(const nsd_config* cfg, void* d_workspace, size_t workspace_bytes, nsd_ctx** out) {
     if (!out) return NSD_ERR_INVALID_ARG;
     *out = nullptr;
     if (!config_ok(cfg) || !d_workspace) return NSD_ERR_INVALID_ARG;
@@ -221,22 +235,13 @@ nsd_status nsd_create(const nsd_config* cfg, void* d_workspace, size_t workspace
     ctx->tmap_slab.assign(cfg->num_slabs, nullptr);
     if ((e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device)) != cudaSuccess) return fail(e, "cudaDeviceGetAttribute");
     ctx->accept_split.n_sms = ctx->n_sms;
-    {
-        // Default: the mma.sync kernel with its K/V tiles fetched by tensor copies where that is the faster feed
-        // (cp.async otherwise).  NSD_ATTN_PATH=mma forces cp.async everywhere, =tcgen05 selects the tcgen05 engine.
-        const char* path = getenv("NSD_ATTN_PATH");
-        ctx->attn_path = !path ? 2 : (strcmp(path, "tcgen05") == 0 ? 1 : (strcmp(path, "mma") == 0 ? 0 : 2));
-    }
-    {
-        // NSD_ROUND_SPLIT=always / never overrides the size rule for the first layer of a round (see round_impl).
-        const char* split = getenv("NSD_ROUND_SPLIT");
-        ctx->round_split = !split ? 0 : (strcmp(split, "always") == 0 ? 1 : (strcmp(split, "never") == 0 ? 2 : 0));
-    }
-    {
-        // NSD_LOGITS_FEED=direct keeps the logits rows on direct loads (the ring of bulk copies is the default).
-        const char* feed = getenv("NSD_LOGITS_FEED");
-        ctx->logits_feed = (feed && strcmp(feed, "direct") == 0) ? 0 : 1;
-    }
+    // Kernel selection (cfg->flags): the defaults are the faster kernel for each shape.
+    ctx->attn_feed_tma = !(cfg->flags & NSD_FLAG_ATTN_CP_ASYNC);
+    ctx->attn_tcgen05 = (cfg->flags & NSD_FLAG_ATTN_NO_TCGEN05) ? 0 : ((cfg->flags & NSD_FLAG_ATTN_TCGEN05) ? 2 : 1);
+    ctx->round_split = (cfg->flags & NSD_FLAG_ROUND_SPLIT_ALWAYS) ? 1 : ((cfg->flags & NSD_FLAG_ROUND_SPLIT_NEVER) ? 2 : 0);
+    ctx->logits_feed = (cfg->flags & NSD_FLAG_LOGITS_DIRECT) ? 0 : 1;
+    ctx->wait_budget = cfg->wait_budget > 0 ? (uint32_t)cfg->wait_budget : 0u;
+    ctx->starve_gather = (cfg->flags & NSD_FLAG_TEST_STARVE_GATHER) ? 16u : 0u;
     *out = ctx;
     return NSD_OK;
 }
@@ -263,9 +268,23 @@ nsd_status nsd_destroy(nsd_ctx* ctx) {
     return NSD_OK;
 }
 
+static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
+                                   const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
+                                   void* stream);
+
 nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
                            const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
                            void* stream) {
+    try {
+        return verify_plan_impl(ctx, batch, gamma, h_ctx_len, h_kv_indptr, h_is_migrated, chunk_blocks, stream);
+    } catch (...) {                        // the host work list could not be allocated: nothing crosses the C boundary
+        return NSD_ERR_CAPACITY;
+    }
+}
+
+static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
+                                   const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
+                                   void* stream) {
     if (!ctx) return NSD_ERR_INVALID_ARG;
     if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
     if (chunk_blocks < 0 || (chunk_blocks & 1) || chunk_blocks > 256) return NSD_ERR_INVALID_ARG;
@@ -381,6 +400,7 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
     ctx->n_res = n_res;
     ctx->n_mig_items = n_all - n_res;
     ctx->plan_src_blocks = src_next;
+    ctx->plan_has_mig = h_is_migrated != nullptr;
     return NSD_OK;
 }
 
@@ -406,7 +426,7 @@ nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
     for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
         uint16_t* slab = slab_ptr(ctx, kv_pool, l);
         if (n_pairs > 0) {
-            NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, mig_src, mig_dst, ctx->d_status, st));
+            NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, mig_src, mig_dst, ctx->d_status, ctx->n_sms, ctx->wait_budget, ctx->starve_gather, st));
             ctx->launches++;
         }
         if (do_append && batch > 0) {
@@ -476,7 +496,8 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
     else if (subset == 1) { a.items = ctx->d_items_split; a.n_items = ctx->n_res; }
     else { a.items = ctx->d_items_split + ctx->n_res; a.n_items = ctx->n_mig_items; }
     if (a.n_items == 0) return NSD_OK;
-    if (ctx->attn_path != 0 && !fuse && ctx->cfg.head_dim == 128) {
+    a.wait_budget = ctx->wait_budget;
+    if ((ctx->attn_feed_tma || ctx->attn_tcgen05) && !fuse && ctx->cfg.head_dim == 128) {
         const int slab = layer % ctx->cfg.num_slabs;
         if (ctx->tmap_slab[slab] != a.pool_slab) {
             ctx->tmap_slab[slab] = make_kv_tensor_map(&ctx->tmaps[slab], a.pool_slab, ctx->shape) ? a.pool_slab : nullptr;
@@ -485,8 +506,8 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
             a.tmap = ctx->tmaps[slab];
             a.tmap_valid = 1;
         }
-        a.tma_feed = ctx->attn_path == 2;
-        if (ctx->attn_path == 1 && attn_umma_supported(a)) {
+        a.tma_feed = ctx->attn_feed_tma;
+        if (ctx->attn_tcgen05 && attn_umma_supported(a) && (ctx->attn_tcgen05 == 2 || attn_umma_preferred(a))) {
             NSD_CUDA(ctx, launch_attn_umma(a, st, ctx->n_sms));
             ctx->launches++;
             return NSD_OK;
@@ -595,7 +616,10 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
     // (tens of microseconds of ramp and tail), so it only pays when the copy is longer than that: from about
     // 60 us of copying (384 MiB read + written) on.  Below, the layer simply waits for its copy.
     const int64_t copy_bytes = n_pairs * ctx->shape.block_elems() * 2 * (int64_t)sizeof(uint16_t);
-    const bool split_first = ctx->round_split == 1 || (ctx->round_split == 0 && copy_bytes >= (384LL << 20));
+    // The split needs the plan's resident / reassigned item lists: a plan made without is_migrated has every request
+    // on the resident list, and attending that list before the copy event would read blocks still being written.
+    const bool can_split = ctx->plan_has_mig && ctx->n_mig_items > 0 && ctx->plan_src_blocks == n_pairs;
+    const bool split_first = can_split && (ctx->round_split == 1 || (ctx->round_split == 0 && copy_bytes >= (384LL << 20)));
     if (overlap) {
         NSD_CUDA(ctx, cudaEventRecord(ctx->ev_start, st));
         NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_start, 0));
@@ -610,7 +634,7 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
             // layer.  The new tokens' rows, which a model only has once it reaches the layer, are appended on the
             // main stream, for every request, right before the layer's attention.
             if (l >= S) NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_attn[l - S], 0));
-            NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, a->mig_src, a->mig_dst, ctx->d_status, ctx->side));
+            NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, a->mig_src, a->mig_dst, ctx->d_status, ctx->n_sms, ctx->wait_budget, ctx->starve_gather, ctx->side));
             NSD_CUDA(ctx, cudaEventRecord(ctx->ev_prep[l], ctx->side));
             ctx->launches++;
             nsd_status s;
@@ -766,7 +790,14 @@ nsd_status nsd_get_status(nsd_ctx* ctx, void* stream, int32_t* first_bad_request
     NSD_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, 4 * sizeof(int32_t), st));
     NSD_CUDA(ctx, cudaStreamSynchronize(st));
     if (first_bad_request) *first_bad_request = ctx->h_status[1] - 1;
-    if (ctx->h_status[0] & STATUS_TIMEOUT) return NSD_ERR_TIMEOUT;
+    if (ctx->h_status[0] & STATUS_TIMEOUT) {
+        // A CTA that gave up never arrived at its request's split-KV counter, so the counter did not return to zero:
+        // clear the arrival counters (attention and acceptance) so that the next launch starts clean.
+        const Layout L = make_layout(&ctx->cfg);
+        NSD_CUDA(ctx, cudaMemsetAsync(ctx->ws + L.counters, 0, L.items_all - L.counters, st));
+        NSD_CUDA(ctx, cudaStreamSynchronize(st));
+        return NSD_ERR_TIMEOUT;
+    }
     if (ctx->h_status[0] & STATUS_LAYOUT) return NSD_ERR_UNSUPPORTED;     // the tcgen05 kernel found its shared memory unaligned
     return ctx->h_status[0] ? NSD_ERR_DEVICE_FAULT : NSD_OK;
 }

@@ -60,11 +60,14 @@ struct AttnLaunch {
     int32_t m_rows;              // (Hq/Hkv) * (gamma+1)
     int32_t tmap_valid;          // tmap describes pool_slab
     int32_t tma_feed;            // mma.sync kernel: fetch K/V tiles with tensor copies where the shape allows
+    uint32_t wait_budget;        // polls per bounded barrier wait, 0 = the kernel's default
     CUtensorMap tmap;
 };
 
+// wait_budget: polls per bounded barrier wait (0 = default); starve_bytes: test hook, extra transaction bytes every
+// barrier expects and never receives (0 in production).
 cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const int32_t* src, const int32_t* dst,
-                          int32_t* status, cudaStream_t stream);
+                          int32_t* status, int n_sms, uint32_t wait_budget, uint32_t starve_bytes, cudaStream_t stream);
 cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int32_t* ctx_len,
                           const int64_t* kv_indptr, const int32_t* kv_indices, const uint16_t* k_new,
                           const uint16_t* v_new, const uint8_t* is_migrated, int32_t subset, int32_t* status,
@@ -77,6 +80,7 @@ cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream);
 cudaError_t gather_init();        // opt in to the copy ring's dynamic shared memory, once per device
 cudaError_t attn_umma_init();     // same for the tcgen05 attention kernels
 bool attn_umma_supported(const AttnLaunch& a);
+bool attn_umma_preferred(const AttnLaunch& a);   // the shapes where the tcgen05 engine is the faster one
 cudaError_t launch_attn_umma(const AttnLaunch& a, cudaStream_t stream, int n_sms);
 bool make_kv_tensor_map(CUtensorMap* map, const void* slab, const Shape& s);
 cudaError_t attn_init();          // opt in to large dynamic shared memory, once per process

@@ -30,7 +30,8 @@ extern "C" nsd_status nsd_schedule_batch(const nsd_sched_params* prm, int32_t n,
     if (!pred_done || !kv_ready || !batch_out) return NSD_ERR_INVALID_ARG;
     if (prm->max_batch < 0 || prm->target_interval < 0 || prm->slack < 0) return NSD_ERR_INVALID_ARG;
 
-    // line 1: filter eligible requests, predict readiness; a request must fit the worker on its own
+    try {
+    // candidate filter: eligible requests with their predicted readiness; a request must fit the worker on its own
     std::vector<Cand> cand;
     cand.reserve(n);
     for (int32_t i = 0; i < n; ++i) {
@@ -45,7 +46,7 @@ extern "C" nsd_status nsd_schedule_batch(const nsd_sched_params* prm, int32_t n,
         c.d = std::max(pred_done[i] + prm->target_interval, c.s_single) + prm->slack;
         cand.push_back(c);
     }
-    // line 2: rank by urgency (admission bound), then predecessor readiness (older output first: the
+    // sort key: urgency (admission bound), then predecessor readiness (older output first: the
     // waiting-time / aging component), then singleton start (temporal compatibility), then index
     std::stable_sort(cand.begin(), cand.end(), [](const Cand& a, const Cand& b) {
         if (a.d != b.d) return a.d < b.d;
@@ -53,10 +54,10 @@ extern "C" nsd_status nsd_schedule_batch(const nsd_sched_params* prm, int32_t n,
         if (a.s_single != b.s_single) return a.s_single < b.s_single;
         return a.idx < b.idx;
     });
-    // line 3: the first at most B_max candidates
+    // only the first B_max candidates are considered
     if ((int64_t)cand.size() > prm->max_batch) cand.resize(prm->max_batch);
 
-    // lines 4-8: greedy admission under Eq. (8)
+    // greedy admission in rank order under Eq. (8)
     double start = prm->worker_avail;     // Eq. (6) of the batch so far: max(a_w, max e, max k)
     double min_d = 0;
     int64_t used_rows = 0, used_blocks = 0, used_tokens = 0;
@@ -79,4 +80,8 @@ extern "C" nsd_status nsd_schedule_batch(const nsd_sched_params* prm, int32_t n,
     *batch_size = m;
     if (batch_start) *batch_start = start;
     return NSD_OK;
+    } catch (...) {                       // the candidate list could not be allocated: nothing crosses the C boundary
+        *batch_size = 0;
+        return NSD_ERR_CAPACITY;
+    }
 }

@@ -109,9 +109,10 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded: gives up after ~2^20 hardware wait slices (seconds); the caller then records STATUS_TIMEOUT and leaves.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < (1u << 20); ++i) {
+// Bounded: gives up after `limit` hardware wait slices (2^20 by default: seconds); the caller then records
+// STATUS_TIMEOUT and leaves.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -189,6 +190,8 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     const int n_total = ctx + gamma + 1;          // keys that exist after the append
     const int M = a.m_rows;
     const int64_t table0 = it.tbl_off >= 0 ? (int64_t)it.tbl_off : a.kv_indptr[r];
+    // a plan checked the table's length on the host; without one (tbl_off < 0) entries past the request's own are not followed
+    const int64_t table_end = it.tbl_off >= 0 ? INT64_MAX : a.kv_indptr[r + 1];
     const int n_blk = it.blk_end - it.blk_begin;
     const int n_tiles = (n_blk + KG - 1) / KG;
 
@@ -201,7 +204,7 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     // ---- block ids of the chunk -> shared (bad ids are replaced by block 0 and reported);
     //      blk_s = where a tile is read from (-1: nowhere, a fresh block), dst_s = where it is written to
     for (int i = tid; i < n_blk; i += NT) {
-        int32_t b = a.kv_indices[table0 + it.blk_begin + i];
+        int32_t b = table0 + it.blk_begin + i < table_end ? a.kv_indices[table0 + it.blk_begin + i] : -1;
         if ((uint32_t)b >= (uint32_t)a.shape.num_blocks) {
             atomicOr(a.status, STATUS_BAD_BLOCK);
             atomicCAS(a.status + 1, 0, r + 1);
@@ -332,12 +335,15 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     // One tile: wait for its copy, refill the stage freed by the previous tile, S^T = K Q^T,
     // online softmax, O^T += V^T P^T.  `stage` is a compile-time constant at every call site.
     bool timed_out = false;                           // TMA-fed variant only: a stage never landed
+    int t_failed = 0;
+    const uint32_t wait_limit = a.wait_budget ? a.wait_budget : (1u << 20);
     auto process_tile = [&](int t, int stage) {
         if constexpr (TMA) {
-            if (!mbar_wait(smem_u32(&full_bar[stage]), (uint32_t)((t / kStages) & 1))) s_timeout = 1;
+            if (!mbar_wait(smem_u32(&full_bar[stage]), (uint32_t)((t / kStages) & 1), wait_limit)) s_timeout = 1;
             __syncthreads();                          // every thread is done with tile t - 1, whose stage is refilled next
             if (s_timeout) {                          // the same answer for every thread of the CTA
                 timed_out = true;
+                t_failed = t;
                 return;
             }
         } else {
@@ -494,7 +500,16 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
             if (t + s < n_tiles && !timed_out) process_tile(t + s, s);
     }
     if (timed_out) {                                      // nothing is written for this item; the status word says why
-        if (tid == 0) atomicOr(a.status, STATUS_TIMEOUT);
+        if (tid == 0) {
+            atomicOr(a.status, STATUS_TIMEOUT);
+            // the tiles armed after the one that never landed may still be arriving in this CTA's shared memory:
+            // give each the same bounded wait before the memory goes back to the SM
+            if constexpr (TMA) {
+                for (int t2 = t_failed + 1; t2 < n_tiles && t2 < t_failed + kStages - 1; ++t2)
+                    mbar_wait(smem_u32(&full_bar[t2 % kStages]), (uint32_t)((t2 / kStages) & 1), wait_limit);
+            }
+        }
+        __syncthreads();
         return;
     }
     cp_async_wait<0>();
@@ -793,11 +808,15 @@ extern "C" nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_bl
         if (n > 1) slots += (int)n;
     }
 
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the work list below is uploaded from this stack frame: a captured copy node would outlive it
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &capturing) != cudaSuccess) return NSD_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone) return NSD_ERR_INVALID_ARG;
     int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return NSD_ERR_CUDA;
     if (static_setup(device) != cudaSuccess) return NSD_ERR_CUDA;
     unsigned char* base = g_static_ptr[device];
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     // The array keeps whatever the previous call left: status and counters must start at zero.
     if (cudaMemsetAsync(base, 0, kStaticOffItems, st) != cudaSuccess) return NSD_ERR_CUDA;
     // The source is pageable (this stack frame): the runtime has staged it when the call returns.

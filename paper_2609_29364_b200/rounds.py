@@ -52,7 +52,7 @@ class RoundRecord:
 
 
 class ScheduledRounds:
-    """`banks` is a workload.banks.BankedPool; `inputs(k, batch)` returns the round's device-side inputs as numpy
+    """`banks` is a BankedPool (banks.py beside this file); `inputs(k, batch)` returns the round's device-side inputs as numpy
     arrays: k_new, v_new, q ([L][rows]...), p, q_draft, draft_tok, u_acc, u_smp."""
 
     def __init__(self, ctx: VerifyContext, kv_pool, banks, ctx_len0: np.ndarray, gamma: int, max_batch: int,

@@ -26,10 +26,14 @@ def host_u16(t: torch.Tensor) -> np.ndarray:
     return t.cpu().numpy().view(np.uint16)
 
 
-def make_context(cfg: W.RoundConfig, meta: W.BatchMeta, num_slabs=None, max_gamma=None):
+CONTEXT_FLAGS = 0                          # nsd_config.flags of the contexts made here; tests that compare kernels patch it
+
+
+def make_context(cfg: W.RoundConfig, meta: W.BatchMeta, num_slabs=None, max_gamma=None, flags=None, wait_budget=0):
     import paper_2609_29364_b200 as nsd
 
-    return nsd.VerifyContext(num_layers=cfg.num_layers, num_slabs=num_slabs or cfg.num_layers,
+    return nsd.VerifyContext(flags=CONTEXT_FLAGS if flags is None else flags, wait_budget=wait_budget,
+                             num_layers=cfg.num_layers, num_slabs=num_slabs or cfg.num_layers,
                              num_q_heads=cfg.num_q_heads, num_kv_heads=cfg.num_kv_heads, head_dim=cfg.head_dim,
                              block_size=cfg.block_size, num_blocks=meta.num_blocks,
                              region_b_begin=meta.region_b_begin, max_batch=cfg.batch,

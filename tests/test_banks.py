@@ -2,7 +2,7 @@
 import numpy as np
 import pytest
 
-from workload.banks import BankedPool
+from paper_2609_29364_b200.banks import BankedPool
 
 
 def _pool():

@@ -1,10 +1,11 @@
 """The mma.sync attention kernel has two ways of fetching K/V tiles: tensor copies (the default where
-the shape is bound by HBM) and cp.async (NSD_ATTN_PATH=mma, and always for the shapes with five or six
+the shape is bound by HBM) and cp.async (NSD_FLAG_ATTN_CP_ASYNC, and always for the shapes with five or six
 row tiles, head_dim 64, gather-through and the allocation-free entry).  Both must match the oracle, and
 each other bit for bit: the feed changes where a tile sits in shared memory, not one operation on it."""
 import numpy as np
 import pytest
 
+import nsd_testlib
 import test_gpu_verify_attn as base
 
 pytestmark = pytest.mark.gpu
@@ -13,7 +14,8 @@ pytestmark = pytest.mark.gpu
 def _both(monkeypatch, cfg, **kw):
     outs = {}
     for feed in ("tma", "mma"):
-        monkeypatch.setenv("NSD_ATTN_PATH", feed)
+        # the tensor-copy feed is the default; neither run may take the tcgen05 engine
+        monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", (1 << 2) | ((1 << 0) if feed == "mma" else 0))
         _, _, o, lse, res = base._run(cfg, want_lse=True, **kw)
         base._check(o, res, lse)
         outs[feed] = (o, lse)

@@ -1,9 +1,10 @@
-"""GPU parity of the tcgen05 / TMEM / TMA attention kernel (opt-in: NSD_ATTN_PATH=tcgen05 when the
-context is created), against the same oracle and tolerance as the default kernel."""
+"""GPU parity of the tcgen05 / TMEM / TMA attention kernel (NSD_FLAG_ATTN_TCGEN05 selects it for
+every shape it supports), against the same oracle and tolerance as the default kernel."""
 import numpy as np
 import pytest
 
 import workload as W
+import nsd_testlib
 import test_gpu_verify_attn as base
 import test_gpu_round as rnd
 
@@ -12,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(autouse=True)
 def _tcgen05_path(monkeypatch):
-    monkeypatch.setenv("NSD_ATTN_PATH", "tcgen05")
+    monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", 1 << 1)
 
 
 @pytest.mark.parametrize("gamma", [1, 4, 6, 8, 11, 15])

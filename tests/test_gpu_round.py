@@ -5,12 +5,15 @@ import numpy as np
 import pytest
 import torch
 
+import nsd_testlib
 import oracle
 import workload as W
 from nsd_testlib import (DeviceBatch, accept_compare, attn_mismatch, dev, guarded_pool, guards_intact, host_u16,
                          make_context, stack_layers)
 
 pytestmark = pytest.mark.gpu
+
+SPLIT_FLAG = {"always": 1 << 4, "never": 1 << 5}      # NSD_FLAG_ROUND_SPLIT_ALWAYS / _NEVER
 
 
 def _oracle_round(cfg, meta, pool0, k_new, v_new, q, acc_in):
@@ -24,8 +27,8 @@ def _oracle_round(cfg, meta, pool0, k_new, v_new, q, acc_in):
     return pool, outs, acc, out, new_ctx
 
 
-def _run_round(cfg, slabs, host_variant=False, repeat=1, fuse=False):
-    """The context reads NSD_ROUND_SPLIT when it is made: the tests below set it to cover both first-layer orders."""
+def _run_round(cfg, slabs, host_variant=False, repeat=1, fuse=False, plan_without_flags=False):
+    """The first-layer order is a flag of the context: the tests below set it to cover both orders."""
     meta = W.make_batch_meta(cfg)
     pool0 = np.stack([W.pool_layer(cfg, meta, s) for s in range(slabs)])
     k_new, v_new = stack_layers(cfg, meta, "kv")
@@ -69,7 +72,8 @@ def _run_round(cfg, slabs, host_variant=False, repeat=1, fuse=False):
         o_gpu, acc_g, out_g, new_g = h["o"].numpy().view(np.uint16), h["acc_len"].numpy(), h["out_tok"].numpy(), h["new_ctx_len"].numpy()
     else:
         with torch.cuda.stream(stream):
-            ctx.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, meta.is_migrated, cfg.gamma, stream=stream)
+            ctx.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, None if plan_without_flags else meta.is_migrated, cfg.gamma,
+                                stream=stream)
             for _ in range(repeat):
                 ctx.nsd_verify_round(ctx.round_args(**d), stream=stream)
         stream.synchronize()
@@ -106,20 +110,20 @@ def test_tiny_config_round():
 def test_multi_layer_round(cfg, slabs, split, monkeypatch):
     """Both orders of the first layer: resident requests attended while the copy runs and the reassigned ones after it
     (what large copies get), or the whole layer after its copy (small copies)."""
-    monkeypatch.setenv("NSD_ROUND_SPLIT", split)
+    monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", SPLIT_FLAG[split])
     _run_round(cfg, slabs)
 
 
 @pytest.mark.parametrize("split", ["always", "never"])
 def test_round_twice_gives_the_same_state(split, monkeypatch):
     """The round is idempotent on its inputs (what the benchmark relies on)."""
-    monkeypatch.setenv("NSD_ROUND_SPLIT", split)
+    monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", SPLIT_FLAG[split])
     _run_round(MULTI, 2, repeat=3)
 
 
 @pytest.mark.parametrize("split", ["always", "never"])
 def test_host_buffer_round(split, monkeypatch):
-    monkeypatch.setenv("NSD_ROUND_SPLIT", split)
+    monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", SPLIT_FLAG[split])
     _run_round(MULTI, 2, host_variant=True)
     _run_round(W.CONFIGS["tiny"], 1, host_variant=True, repeat=2)
 
@@ -157,9 +161,18 @@ def test_gather_through_needs_a_matching_plan():
     assert e.value.code == 1 and ctx.nsd_launch_count() == 0
 
 
+def test_round_with_a_plan_made_without_the_reassignment_flags(monkeypatch):
+    """Such a plan has every request on its resident list: the round must not attend that list before the copy has
+    finished, even when the context is told to split its first layer."""
+    monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", SPLIT_FLAG["always"])
+    ctx = _run_round(MULTI, 2, plan_without_flags=True)
+    assert ctx.nsd_launch_count() == MULTI.num_layers * 3 + 1            # no second attention launch in the first layer
+    _run_round(ALLMIG, 3, plan_without_flags=True, repeat=2)
+
+
 def test_launch_count_matches_the_choreography(monkeypatch):
     # per layer: the copy (side stream), one append and one attention launch; one acceptance
     assert _run_round(MULTI, 5).nsd_launch_count() == 5 * 3 + 1          # a small copy: the first layer waits for it
-    monkeypatch.setenv("NSD_ROUND_SPLIT", "always")
+    monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", SPLIT_FLAG["always"])
     # the first layer appends and attends its resident and its reassigned requests separately: two launches more
     assert _run_round(MULTI, 5).nsd_launch_count() == 5 * 3 + 2 + 1

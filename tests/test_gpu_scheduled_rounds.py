@@ -9,7 +9,7 @@ import torch
 import oracle
 import workload as W
 from oracle import schedule as osched
-from workload.banks import BankedPool
+from paper_2609_29364_b200.banks import BankedPool
 from nsd_testlib import accept_compare, attn_mismatch, host_u16
 
 pytestmark = pytest.mark.gpu

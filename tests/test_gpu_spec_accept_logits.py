@@ -8,6 +8,7 @@ from scipy.special import softmax
 
 import oracle
 import workload as W
+import nsd_testlib
 from nsd_testlib import TOKEN_CDF_TOL, dev, make_context
 from workload.gen import uniforms
 
@@ -140,7 +141,7 @@ def test_qwen3_vocab_bf16_logits():
 @pytest.mark.parametrize("B", [200, 320], ids=["deep_ring", "four_per_sm"])
 @pytest.mark.parametrize("V,dtype,T", [(4104, 0, 0.8), (20488, 0, 1.0), (8200, 1, 1.0), (12296, 1, 0.0), (2052, 0, 0.0)])
 def test_ring_and_direct_feeds_agree_bit_for_bit(V, dtype, T, B, monkeypatch):
-    """Rows whose starts are 16-byte aligned travel through the shared-memory ring of bulk copies; NSD_LOGITS_FEED=direct
+    """Rows whose starts are 16-byte aligned travel through the shared-memory ring of bulk copies; NSD_FLAG_LOGITS_DIRECT
     keeps them on direct loads.  Every thread sees the same elements in the same order, so nothing may differ.  The
     vocabularies span several 8 KiB tiles with a ragged last one, both for the row sweep and for the draw."""
     # batch 200: CTAs have an SM (nearly) to themselves and get the 12-tile ring; batch 320: four CTAs per SM, 4 tiles
@@ -156,7 +157,7 @@ def test_ring_and_direct_feeds_agree_bit_for_bit(V, dtype, T, B, monkeypatch):
         tok[wrong] = (tok[wrong] + 3) % V
     res = {}
     for feed in ("ring", "direct"):
-        monkeypatch.setenv("NSD_LOGITS_FEED", feed)
+        monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", (1 << 3) if feed == "direct" else 0)
         res[feed] = _gpu(z, dtype, T, q, tok, ua, us) if T > 0 else _gpu(z, dtype, 0.0, None, tok, None, None)
     assert np.array_equal(res["ring"][0], res["direct"][0]) and np.array_equal(res["ring"][1], res["direct"][1])
     acc_r, out_r, _ = oracle.spec_accept_logits(z, T, q, tok, ua, us) if T > 0 else oracle.spec_accept_logits(z, 0.0, None, tok, None, None)

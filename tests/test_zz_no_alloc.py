@@ -1,15 +1,16 @@
 """nsd_verify_attn_static: attention for hosts that may not allocate device memory
 (a plugin inside another runtime's memory budget, a worker whose memory was carved
 up at start-up).  Its scratch is a fixed array inside the library, so the checks
-that matter are: same output as the workspace-backed nsd_verify_attn, still the
-same on a second call that finds the first call's leftovers in the array, and a
-clean refusal of batches that exceed the array.
+that matter are: same output as the workspace-backed nsd_verify_attn and as the
+oracle, still the same on a second call that finds the first call's leftovers in
+the array, and a clean refusal of batches that exceed the array.
 
 Collected last on purpose (file name): a failure here cannot hide the other tests."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import workload as W
 from nsd_testlib import DeviceBatch, attn_mismatch, dev, host_u16, make_context
 
@@ -33,7 +34,11 @@ def _case(seed, ctx):
     ctxh.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, None, cfg.gamma)
     ctxh.nsd_verify_attn(pool_d, q_d, o_ref, None, cfg.batch, cfg.gamma, db.ctx_len, db.kv_indptr, db.kv_indices)
     torch.cuda.synchronize()
-    return cfg, meta, db, pool_d, q_d, o_ref
+    # the oracle on the same prepared pool
+    want = pool[None].copy()
+    oracle.kv_prepare(want, None, None, None, meta.ctx_len, meta.kv_indptr, meta.kv_indices, k_new[None], v_new[None], cfg.gamma)
+    o_oracle = oracle.verify_attn(want, q, meta.ctx_len, meta.kv_indptr, meta.kv_indices, cfg.gamma)
+    return cfg, meta, db, pool_d, q_d, o_ref, o_oracle
 
 
 def _static(cfg, meta, db, pool_d, q_d):
@@ -51,17 +56,19 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     first = _case(91, [3, 200, 1023, 1500, 2500, 40])        # two split requests: 2 and 3 chunks
     second = _case(92, [3000, 17, 1100, 900])                 # other lengths: other chunk counts per slot
     for case in (first, second, first):
-        cfg, meta, db, pool_d, q_d, o_ref = case
+        cfg, meta, db, pool_d, q_d, o_ref, o_oracle = case
         o = _static(cfg, meta, db, pool_d, q_d)
         ref = W.bf16_to_f32(host_u16(o_ref))
         bad, max_abs, max_rel = attn_mismatch(host_u16(o), ref)
+        assert bad == 0, (bad, max_abs, max_rel)
+        bad, max_abs, max_rel = attn_mismatch(host_u16(o), o_oracle)
         assert bad == 0, (bad, max_abs, max_rel)
 
 
 def test_sizes_beyond_the_static_scratch_are_refused():
     import paper_2609_29364_b200 as nsd
 
-    cfg, meta, db, pool_d, q_d, o_ref = _case(93, [10, 20])
+    cfg, meta, db, pool_d, q_d, o_ref, _ = _case(93, [10, 20])
     o = torch.zeros_like(q_d)
     common = (pool_d, meta.num_blocks, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.block_size, q_d, o)
     tables = (db.ctx_len, db.kv_indptr, db.kv_indices)
@@ -79,3 +86,20 @@ def test_sizes_beyond_the_static_scratch_are_refused():
     assert e.value.code == 1
     torch.cuda.synchronize()
     assert (o == 0).all()                                     # nothing was launched
+
+
+def test_a_capturing_stream_is_refused():
+    """The call uploads its work list from a buffer that dies with the call, so it cannot become a graph node."""
+    import paper_2609_29364_b200 as nsd
+
+    cfg, meta, db, pool_d, q_d, o_ref, _ = _case(94, [10, 20])
+    _static(cfg, meta, db, pool_d, q_d)                        # the set-up call, outside any capture
+    o = torch.zeros_like(q_d)
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        with pytest.raises(nsd.NsdError) as e:
+            nsd.nsd_verify_attn_static(pool_d, meta.num_blocks, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim,
+                                       cfg.block_size, q_d, o, cfg.batch, cfg.gamma, meta.ctx_len, db.ctx_len,
+                                       db.kv_indptr, db.kv_indices, stream=stream)
+        assert e.value.code == 1

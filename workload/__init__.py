@@ -18,6 +18,7 @@ from .gen import (  # noqa: F401
     make_batch_meta,
     new_kv,
     pool_layer,
+    pool_layer_chunks,
     queries,
     BF16_NAN,
 )

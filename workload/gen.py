@@ -112,7 +112,7 @@ class RoundConfig:
 _QWEN = dict(num_q_heads=32, num_kv_heads=8, head_dim=128, block_size=16, vocab=151936)
 
 CONFIGS = {
-    # benchmark configs[0..4], in order
+    # the five configurations of the benchmark set, in order
     "tiny": RoundConfig("tiny", batch=4, gamma=4, num_layers=1, num_q_heads=8, num_kv_heads=2, head_dim=64,
                         block_size=16, vocab=1000, ctx_dist=("uniform", 17, 100), frac_reassigned=0.25,
                         noise_var=None, seed=20260929),
@@ -218,6 +218,28 @@ def make_batch_meta(cfg: RoundConfig) -> BatchMeta:
 
 
 # --------------------------------------------------------------------------- per-layer tensors
+def pool_layer_chunks(cfg: RoundConfig, meta: BatchMeta, layer: int, poison: bool = True, step: int = 1024):
+    """The committed KV of one layer slab, streamed: yields (b0, b1, data) where `data`
+    (uint16 [b1-b0][2][num_kv_heads][block_size][head_dim]) is the content of home blocks
+    `meta.home_blocks[b0:b1]`, tail slots of a request's last block already filled.  The
+    draws are those of `pool_layer` (one stream, `step` home blocks per draw), so a slab far
+    larger than host memory can be produced -- or re-read -- piece by piece."""
+    Hkv, bs, D = cfg.num_kv_heads, cfg.block_size, cfg.head_dim
+    fill = BF16_NAN if poison else np.uint16(0)
+    n_home = int(meta.home_indptr[-1])
+    rng = _rng(cfg.seed, "pool", layer)
+    tail = meta.ctx_len.astype(np.int64) % bs
+    last_of = meta.home_indptr[1:] - 1                 # home index of each request's last block
+    tailed = np.nonzero(tail)[0]
+    assert step == 1024, "the draw size is part of the recipe: it fixes the stream"
+    for b0 in range(0, n_home, step):
+        b1 = min(n_home, b0 + step)
+        data = _normal_bf16(rng, (b1 - b0, 2, Hkv, bs, D))
+        for r in tailed[(last_of[tailed] >= b0) & (last_of[tailed] < b1)]:
+            data[int(last_of[r]) - b0, :, :, int(tail[r]):, :] = fill
+        yield b0, b1, data
+
+
 def pool_layer(cfg: RoundConfig, meta: BatchMeta, layer: int, poison: bool = True) -> np.ndarray:
     """One layer slab of the paged pool before the round, bf16 bits as uint16,
     shape [num_blocks][2 (K,V)][num_kv_heads][block_size][head_dim].
@@ -230,17 +252,8 @@ def pool_layer(cfg: RoundConfig, meta: BatchMeta, layer: int, poison: bool = Tru
     Hkv, bs, D = cfg.num_kv_heads, cfg.block_size, cfg.head_dim
     fill = BF16_NAN if poison else np.uint16(0)
     pool = np.full((meta.num_blocks, 2, Hkv, bs, D), fill, dtype=np.uint16)
-    n_home = int(meta.home_indptr[-1])
-    if n_home:
-        rng = _rng(cfg.seed, "pool", layer)
-        step = 1024                                   # home blocks per draw (part of the recipe: fixes the stream)
-        for b0 in range(0, n_home, step):
-            b1 = min(n_home, b0 + step)
-            pool[meta.home_blocks[b0:b1]] = _normal_bf16(rng, (b1 - b0, 2, Hkv, bs, D))
-        tail = meta.ctx_len.astype(np.int64) % bs
-        for r in np.nonzero(tail)[0]:
-            last = int(meta.home_blocks[int(meta.home_indptr[r + 1]) - 1])
-            pool[last, :, :, int(tail[r]):, :] = fill
+    for b0, b1, data in pool_layer_chunks(cfg, meta, layer, poison):
+        pool[meta.home_blocks[b0:b1]] = data
     return pool
 
 
