@@ -52,6 +52,7 @@ def parse_args():
     ap.add_argument("--no-scheduled", action="store_true", help="skip the scheduler-driven two-bank rounds leg")
     ap.add_argument("--scheduled-rounds", type=int, default=8)
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target CPU time of the oracle sample")
+    ap.add_argument("--ctx-flags", type=int, default=0, help="comparison runs only: nsd_config.flags of the context (not a bench line)")
     ap.add_argument("--batch", type=int, default=0, help="profiling only: override the batch size (not a bench line)")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: override the layer count (not a bench line)")
     return ap.parse_args()
@@ -348,7 +349,7 @@ def run_ours(args):
     ctx = nsd.VerifyContext(num_layers=L, num_slabs=slabs, num_q_heads=cfg.num_q_heads, num_kv_heads=cfg.num_kv_heads,
                             head_dim=cfg.head_dim, block_size=cfg.block_size, num_blocks=meta.num_blocks,
                             region_b_begin=meta.region_b_begin, max_batch=B, max_gamma=cfg.gamma, vocab_size=cfg.vocab,
-                            max_table_entries=int(meta.kv_indptr[-1]), device=str(device))
+                            max_table_entries=int(meta.kv_indptr[-1]), flags=args.ctx_flags, device=str(device))
     pool = torch.empty((slabs, meta.num_blocks * cfg.block_elems), dtype=torch.int16, device=device)
     pool[0].copy_(torch.from_numpy(host["pool_slab"].reshape(-1).view(np.int16)))
     for s in range(1, slabs):

@@ -36,6 +36,7 @@ struct nsd_ctx {
     bool planned;
     int32_t plan_batch, plan_gamma;
     int32_t n_all, n_res, n_mig_items;
+    int32_t plan_split_slots;  // partial slots the plan uses (0 = no request is split)
     int64_t plan_src_blocks;   // source blocks of the planned batch's reassigned requests
     bool plan_has_mig;         // the plan was given is_migrated (its resident / reassigned item lists are meaningful)
     // streams / events
@@ -45,8 +46,9 @@ struct nsd_ctx {
     std::vector<cudaEvent_t> ev_prep, ev_attn;
     std::vector<cudaEvent_t> ev_in, ev_out;    // nsd_verify_round_host: layer l's inputs have landed / its output is complete
     // tcgen05 attention: one tensor map per layer slab of the pool last seen, and the SM count for the persistent grid
-    std::vector<CUtensorMap> tmaps;
+    std::vector<CUtensorMap> tmaps, tmaps3;
     std::vector<const void*> tmap_slab;
+    std::vector<char> tmap3_ok;
     int n_sms;
     int round_split;           // first layer of a round with reassigned requests: 0 = by size, 1 = always attend resident and reassigned requests separately, 2 = never
     int logits_feed;           // acceptance from logits: 1 = rows through the shared-memory ring where aligned (default), 0 = direct loads
@@ -232,6 +234,8 @@ static nsd_status create_impl(const nsd_config* cfg, void* d_workspace, size_t w
     if ((e = gather_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(gather)");
     if ((e = attn_umma_init()) != cudaSuccess) return fail(e, "cudaFuncSetAttribute(tcgen05 attention)");
     ctx->tmaps.resize(cfg->num_slabs);
+    ctx->tmaps3.resize(cfg->num_slabs);
+    ctx->tmap3_ok.assign(cfg->num_slabs, 0);
     ctx->tmap_slab.assign(cfg->num_slabs, nullptr);
     if ((e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device)) != cudaSuccess) return fail(e, "cudaDeviceGetAttribute");
     ctx->accept_split.n_sms = ctx->n_sms;
@@ -400,6 +404,7 @@ static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, c
     ctx->n_res = n_res;
     ctx->n_mig_items = n_all - n_res;
     ctx->plan_src_blocks = src_next;
+    ctx->plan_split_slots = slot;
     ctx->plan_has_mig = h_is_migrated != nullptr;
     return NSD_OK;
 }
@@ -497,19 +502,25 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
     else { a.items = ctx->d_items_split + ctx->n_res; a.n_items = ctx->n_mig_items; }
     if (a.n_items == 0) return NSD_OK;
     a.wait_budget = ctx->wait_budget;
+    a.any_split = ctx->plan_split_slots > 0;
     if ((ctx->attn_feed_tma || ctx->attn_tcgen05) && !fuse && ctx->cfg.head_dim == 128) {
         const int slab = layer % ctx->cfg.num_slabs;
         if (ctx->tmap_slab[slab] != a.pool_slab) {
             ctx->tmap_slab[slab] = make_kv_tensor_map(&ctx->tmaps[slab], a.pool_slab, ctx->shape) ? a.pool_slab : nullptr;
+            ctx->tmap3_ok[slab] = ctx->attn_tcgen05 && ctx->tmap_slab[slab] && make_kv_tensor_map3(&ctx->tmaps3[slab], a.pool_slab, ctx->shape);
         }
         if (ctx->tmap_slab[slab] == a.pool_slab) {
             a.tmap = ctx->tmaps[slab];
             a.tmap_valid = 1;
+            if (ctx->tmap3_ok[slab]) {
+                a.tmap3 = ctx->tmaps3[slab];
+                a.tmap3_valid = 1;
+            }
         }
         a.tma_feed = ctx->attn_feed_tma;
         if (ctx->attn_tcgen05 && attn_umma_supported(a) && (ctx->attn_tcgen05 == 2 || attn_umma_preferred(a))) {
             NSD_CUDA(ctx, launch_attn_umma(a, st, ctx->n_sms));
-            ctx->launches++;
+            ctx->launches += a.any_split ? 2 : 1;                            // the engine's merge kernel follows when a request is split
             return NSD_OK;
         }
     }

@@ -61,7 +61,10 @@ struct AttnLaunch {
     int32_t tmap_valid;          // tmap describes pool_slab
     int32_t tma_feed;            // mma.sync kernel: fetch K/V tiles with tensor copies where the shape allows
     uint32_t wait_budget;        // polls per bounded barrier wait, 0 = the kernel's default
+    int32_t tmap3_valid;         // tmap3 describes pool_slab
+    int32_t any_split;           // some request of the plan has more than one chunk (the tcgen05 engine then launches its merge)
     CUtensorMap tmap;
+    CUtensorMap tmap3;           // tcgen05 engine: 3-D view whose box is a block's whole [16 keys][128 dims] tile
 };
 
 // wait_budget: polls per bounded barrier wait (0 = default); starve_bytes: test hook, extra transaction bytes every
@@ -83,6 +86,7 @@ bool attn_umma_supported(const AttnLaunch& a);
 bool attn_umma_preferred(const AttnLaunch& a);   // the shapes where the tcgen05 engine is the faster one
 cudaError_t launch_attn_umma(const AttnLaunch& a, cudaStream_t stream, int n_sms);
 bool make_kv_tensor_map(CUtensorMap* map, const void* slab, const Shape& s);
+bool make_kv_tensor_map3(CUtensorMap* map, const void* slab, const Shape& s);
 cudaError_t attn_init();          // opt in to large dynamic shared memory, once per process
 // Scratch for sharing one request among several acceptance CTAs (small batches): one row of segment sums and one
 // arrival counter (zero between launches) per request.
