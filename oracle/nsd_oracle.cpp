@@ -79,6 +79,23 @@ struct PoolShape {
     }
 };
 
+// Rows per request when drafts are ragged (Appendix G.2 studies draft depths 3, 4, 5: the target verifies "anchor plus
+// proposal" tokens of each request, and a batch may mix depths).  Request r brings gamma_r[r] proposals, so gamma_r[r] + 1
+// rows; its rows start at the sum of the rows before it.  With gamma_r == nullptr every request has gamma + 1 rows.
+// Returns false when a depth lies outside [0, gamma].
+bool row_offsets(int batch, int gamma, const int32_t* gamma_r, std::vector<int64_t>& row0, std::vector<int>& depth) {
+    row0.assign(batch + 1, 0);
+    depth.assign(batch, gamma);
+    for (int r = 0; r < batch; ++r) {
+        if (gamma_r) {
+            if (gamma_r[r] < 0 || gamma_r[r] > gamma) return false;
+            depth[r] = gamma_r[r];
+        }
+        row0[r + 1] = row0[r] + depth[r] + 1;
+    }
+    return true;
+}
+
 }  // namespace
 
 extern "C" {
@@ -90,18 +107,21 @@ int oracle_hardware_threads() {
 
 // Gather, then append, one logical layer after the other.  Logical layer l
 // lives in physical slab l % num_slabs.  k_new / v_new are indexed by logical
-// layer: [num_layers][rows][Hkv][D]; pass nullptr to skip the append.
+// layer: [num_layers][rows][Hkv][D]; pass nullptr to skip the append.  gamma_r
+// (nullable): per-request draft depth, rows ragged (see row_offsets).
 // Returns 0, or a negative code when an index leaves its range (nothing is
 // written for that item).
 int oracle_kv_prepare(uint16_t* pool, int num_slabs, int64_t num_blocks, int Hkv, int bs, int D,
                       int n_mig, const int64_t* mig_indptr, const int32_t* mig_src, const int32_t* mig_dst,
                       int batch, int gamma, const int32_t* ctx_len, const int64_t* kv_indptr,
                       const int32_t* kv_indices, const uint16_t* k_new, const uint16_t* v_new,
-                      int layer_begin, int layer_count) {
+                      int layer_begin, int layer_count, const int32_t* gamma_r) {
     PoolShape ps{num_blocks, Hkv, bs, D};
     const int64_t blk = ps.block_elems();
-    const int rows_per_req = gamma + 1;
-    const int64_t layer_rows = static_cast<int64_t>(batch) * rows_per_req;
+    std::vector<int64_t> row0;
+    std::vector<int> depth;
+    if (!row_offsets(batch, gamma, gamma_r, row0, depth)) return -7;
+    const int64_t layer_rows = row0[batch];
     int rc = 0;
     for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
         const int64_t slab = l % num_slabs;
@@ -116,14 +136,14 @@ int oracle_kv_prepare(uint16_t* pool, int num_slabs, int64_t num_blocks, int Hkv
         if (!k_new || !v_new) continue;
         // append: token t of request r goes to position ctx_r + t
         for (int r = 0; r < batch; ++r)
-            for (int t = 0; t < rows_per_req; ++t) {
+            for (int t = 0; t <= depth[r]; ++t) {
                 int64_t pos = static_cast<int64_t>(ctx_len[r]) + t;
                 int64_t entry = kv_indptr[r] + pos / bs;
                 if (ctx_len[r] < 0 || entry >= kv_indptr[r + 1]) { rc = -2; continue; }
                 int64_t b = kv_indices[entry];
                 if (b < 0 || b >= num_blocks) { rc = -1; continue; }
                 int slot = static_cast<int>(pos % bs);
-                int64_t row = static_cast<int64_t>(l) * layer_rows + static_cast<int64_t>(r) * rows_per_req + t;
+                int64_t row = static_cast<int64_t>(l) * layer_rows + row0[r] + t;
                 for (int h = 0; h < Hkv; ++h) {
                     std::memcpy(pool + ps.at(slab, b, 0, h, slot, 0), k_new + (row * Hkv + h) * D, D * sizeof(uint16_t));
                     std::memcpy(pool + ps.at(slab, b, 1, h, slot, 0), v_new + (row * Hkv + h) * D, D * sizeof(uint16_t));
@@ -142,13 +162,13 @@ int oracle_kv_prepare(uint16_t* pool, int num_slabs, int64_t num_blocks, int Hkv
 int oracle_kv_commit(uint16_t* pool, int num_slabs, int64_t num_blocks, int Hkv, int bs, int D, int batch, int gamma,
                      const int32_t* ctx_len, const int32_t* acc_len, const int64_t* kv_indptr,
                      const int32_t* kv_indices, const int64_t* exp_indptr, const int32_t* exp_indices,
-                     int32_t* new_ctx_len, int layer_begin, int layer_count) {
+                     int32_t* new_ctx_len, int layer_begin, int layer_count, const int32_t* gamma_r) {
     PoolShape ps{num_blocks, Hkv, bs, D};
     int rc = 0;
     for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
         const int64_t slab = l % num_slabs;
         for (int r = 0; r < batch; ++r) {
-            if (acc_len[r] < 0 || acc_len[r] > gamma) { rc = -6; continue; }
+            if (acc_len[r] < 0 || acc_len[r] > (gamma_r ? gamma_r[r] : gamma)) { rc = -6; continue; }   // at most the drafts it had
             for (int t = 0; t <= acc_len[r]; ++t) {
                 const int64_t pos = static_cast<int64_t>(ctx_len[r]) + t;
                 const int64_t from = kv_indices[kv_indptr[r] + pos / bs], to = exp_indices[exp_indptr[r] + pos / bs];
@@ -172,8 +192,11 @@ int oracle_kv_commit(uint16_t* pool, int num_slabs, int64_t num_blocks, int Hkv,
 int oracle_verify_attn(const uint16_t* pool, int num_slabs, int64_t num_blocks, int Hq, int Hkv, int bs, int D,
                        const uint16_t* q, float* o, float* lse, int batch, int gamma, const int32_t* ctx_len,
                        const int64_t* kv_indptr, const int32_t* kv_indices, int layer,
-                       const int32_t* req_list, int n_req, int nthreads) {
+                       const int32_t* req_list, int n_req, int nthreads, const int32_t* gamma_r) {
     if (Hkv <= 0 || Hq % Hkv != 0) return -3;
+    std::vector<int64_t> row0;
+    std::vector<int> depth;
+    if (!row_offsets(batch, gamma, gamma_r, row0, depth)) return -7;
     PoolShape ps{num_blocks, Hkv, bs, D};
     const int group = Hq / Hkv;
     const int64_t slab = layer % num_slabs;
@@ -184,9 +207,9 @@ int oracle_verify_attn(const uint16_t* pool, int num_slabs, int64_t num_blocks, 
         const int r = req_list ? req_list[it] : static_cast<int>(it);
         if (r < 0 || r >= batch) { rc = -4; return; }
         std::vector<double> s, acc(D);
-        for (int i = 0; i <= gamma; ++i) {
+        for (int i = 0; i <= depth[r]; ++i) {
             const int64_t n_keys = static_cast<int64_t>(ctx_len[r]) + i + 1;
-            const int64_t row = static_cast<int64_t>(r) * (gamma + 1) + i;
+            const int64_t row = row0[r] + i;
             s.resize(n_keys);
             for (int h = 0; h < Hq; ++h) {
                 const int g = h / group;
@@ -218,25 +241,36 @@ int oracle_verify_attn(const uint16_t* pool, int num_slabs, int64_t num_blocks, 
     return rc;
 }
 
-// Acceptance.  p: [batch][gamma+1][V], q: [batch][gamma][V], fp32.  All
+// Acceptance.  p: [batch][gamma+1][V], q: [batch][gamma][V], fp32 -- or, with gamma_r
+// (per-request draft depth), ragged: gamma_r[r] + 1 target rows, gamma_r[r] draft rows,
+// draft tokens and accept uniforms, gamma_r[r] + 1 output tokens per request.  All
 // compares and sums in double on the fp32 inputs; the residual p - q is an fp32
 // subtraction, then widened.  out_tok: [batch][gamma+1] = accepted drafts, the
 // resampled or bonus token, then -1 padding.
 int oracle_spec_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
                        const float* u_smp, int batch, int gamma, int64_t vocab, const int32_t* ctx_len,
-                       int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int nthreads) {
+                       int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int nthreads, const int32_t* gamma_r) {
     std::atomic<int> rc{0};
+    std::vector<int64_t> row0;
+    std::vector<int> depth;
+    if (!row_offsets(batch, gamma, gamma_r, row0, depth)) return -7;
     parallel_for(batch, nthreads, [&](int64_t r) {
-        const float* pr = p + r * (gamma + 1) * vocab;
-        const float* qr = q + r * gamma * vocab;
+        // target rows start at row0[r]; the request has one draft row fewer than target rows, so its draft rows, draft
+        // tokens and accept uniforms start at row0[r] - r
+        const int gamma = depth[r];
+        const int64_t d0 = row0[r] - r;
+        const float* pr = p + row0[r] * vocab;
+        const float* qr = q + d0 * vocab;
+        const int32_t* draft_tok_r = draft_tok + d0;
+        const float* u_acc_r = u_acc + d0;
         int n = gamma;
         for (int i = 0; i < gamma; ++i) {
-            int32_t x = draft_tok[r * gamma + i];
+            int32_t x = draft_tok_r[i];
             if (x < 0 || x >= vocab) { rc = -5; n = i; break; }
             double P = pr[i * vocab + x], Q = qr[i * vocab + x];
             double ratio = (Q > 0.0) ? P / Q : (P > 0.0 ? 1.0 : 0.0);
             double thr = ratio < 1.0 ? ratio : 1.0;
-            if (!(static_cast<double>(u_acc[r * gamma + i]) < thr)) { n = i; break; }
+            if (!(static_cast<double>(u_acc_r[i]) < thr)) { n = i; break; }
         }
         const float* prow = pr + static_cast<int64_t>(n) * vocab;
         std::vector<double> w(vocab);
@@ -263,8 +297,8 @@ int oracle_spec_accept(const float* p, const float* q, const int32_t* draft_tok,
         }
         if (y < 0) y = last_pos;
         acc_len[r] = n;
-        int32_t* out = out_tok + r * (gamma + 1);
-        for (int i = 0; i <= gamma; ++i) out[i] = i < n ? draft_tok[r * gamma + i] : (i == n ? static_cast<int32_t>(y) : -1);
+        int32_t* out = out_tok + row0[r];
+        for (int i = 0; i <= gamma; ++i) out[i] = i < n ? draft_tok_r[i] : (i == n ? static_cast<int32_t>(y) : -1);
         if (new_ctx_len && ctx_len) new_ctx_len[r] = ctx_len[r] + 1 + n;
     });
     return rc;

@@ -13,6 +13,8 @@ from .gen import (  # noqa: F401
     accept_inputs,
     bf16_to_f32,
     draw_ctx_len,
+    draw_gamma_r,
+    ragged_index,
     export_tables,
     f32_to_bf16,
     make_batch_meta,

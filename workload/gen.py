@@ -337,3 +337,22 @@ def accept_inputs(cfg: RoundConfig, batch: Optional[int] = None, chunk: int = 16
     u_acc = uniforms(_rng(cfg.seed, "u_acc"), (B, g))
     u_smp = uniforms(_rng(cfg.seed, "u_smp"), (B,))
     return p, q, tok, u_acc, u_smp
+
+
+# --------------------------------------------------------------------------- per-request draft depth
+def draw_gamma_r(cfg: RoundConfig, lo: int = 0) -> np.ndarray:
+    """Per-request draft depth in [lo, cfg.gamma] (int32 [batch]): a batch that mixes depths, as when requests come from
+    draft workers run at different depths."""
+    return _rng(cfg.seed, "ctx", 99).integers(lo, cfg.gamma + 1, size=cfg.batch).astype(np.int32)
+
+
+def ragged_index(gamma_r: np.ndarray, gamma: int):
+    """Indices that cut padded per-request tensors down to their ragged form: `rows` picks entries (r, i <= gamma_r[r]) out
+    of [batch*(gamma+1)] target rows, `drafts` picks (r, i < gamma_r[r]) out of [batch*gamma] draft rows; `row_indptr`
+    (int64 [batch+1]) is the prefix of gamma_r + 1."""
+    B = len(gamma_r)
+    rows = np.concatenate([r * (gamma + 1) + np.arange(gamma_r[r] + 1) for r in range(B)]).astype(np.int64)
+    drafts = np.concatenate([r * gamma + np.arange(gamma_r[r]) for r in range(B)] + [np.zeros(0, np.int64)]).astype(np.int64)
+    row_indptr = np.zeros(B + 1, dtype=np.int64)
+    np.cumsum(gamma_r.astype(np.int64) + 1, out=row_indptr[1:])
+    return rows, drafts, row_indptr
