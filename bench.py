@@ -497,6 +497,28 @@ def run_ours(args):
     ms_round_fused = timed(lambda: ctx.nsd_verify_round(fused_args, stream=stream), args.steps, args.warmup)
     assert np.array_equal(d["acc_len"].cpu().numpy(), acc_len)
 
+    # ---- a batch that mixes draft depths (ragged rows) against the same batch padded to the deepest draft
+    gamma_r = W.draw_gamma_r(cfg, lo=(cfg.gamma + 1) // 2)
+    rows_idx, drafts_idx, q_indptr = W.ragged_index(gamma_r, cfg.gamma)
+    ri, di = torch.from_numpy(rows_idx).to(device), torch.from_numpy(drafts_idx).to(device)
+    V = cfg.vocab
+    rag = dict(d)
+    rag.update(k_new=d["k_new"][:, ri].contiguous(), v_new=d["v_new"][:, ri].contiguous(), q=d["q"][:, ri].contiguous(),
+               o=torch.zeros((L, len(rows_idx)) + tuple(d["q"].shape[2:]), dtype=torch.int16, device=device),
+               p=d["p"].reshape(-1, V)[ri].contiguous(), q_draft=d["q_draft"].reshape(-1, V)[di].contiguous(),
+               draft_tok=d["draft_tok"].reshape(-1)[di].contiguous(), u_acc=d["u_acc"].reshape(-1)[di].contiguous(),
+               out_tok=torch.zeros(len(rows_idx), dtype=torch.int32, device=device), q_indptr=dev(q_indptr))
+    with torch.cuda.stream(stream):
+        ctx.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, meta.is_migrated, cfg.gamma, stream=stream, h_q_indptr=q_indptr)
+    rag_args = ctx.round_args(**rag)
+    ms_round_ragged = timed(lambda: ctx.nsd_verify_round(rag_args, stream=stream), args.steps, args.warmup)
+    rc, bad = ctx.nsd_get_status(stream=stream)
+    if rc != 0:
+        raise SystemExit(f"device status {rc} (request {bad}) in the mixed-depth round")
+    del rag, rag_args
+    with torch.cuda.stream(stream):
+        ctx.nsd_verify_plan(meta.ctx_len, meta.kv_indptr, meta.is_migrated, cfg.gamma, stream=stream)
+
     # ---- end to end: per-round tensors start in pinned host memory, results read back
     e2e = None
     if not args.no_e2e:
@@ -593,6 +615,13 @@ def run_ours(args):
                 "algorithmic_bytes_per_round": bytes_["round"] - L * bytes_["gather_per_layer"] // 2,
                 "achieved_GBs": (bytes_["round"] - L * bytes_["gather_per_layer"] // 2) / (ms_round_fused * 1e-3) / 1e9,
                 "speedup_over_headline": ms_round / ms_round_fused},
+            "mixed_depth_round": {
+                "what": "the same batch with per-request draft depths drawn from [%d, %d] (ragged rows, one attention launch per "
+                        "row-tile class) against the batch padded to depth %d, which is the headline round" % ((cfg.gamma + 1) // 2, cfg.gamma, cfg.gamma),
+                "rows": int(len(rows_idx)), "padded_rows": int(cfg.rows), "ms_per_step": ms_round_ragged,
+                "useful_rows_per_s": n_gpus * len(rows_idx) / (ms_round_ragged * 1e-3),
+                "useful_rows_per_s_padded": n_gpus * len(rows_idx) / (ms_round * 1e-3),
+                "speedup_over_padded": ms_round / ms_round_ragged},
             "round_cuda_graph": None if ms_round_graph is None else {
                 "ms_per_step": ms_round_graph, "value": n_gpus * B / (ms_round_graph * 1e-3), "unit": "req/s"},
             "scheduled_rounds": scheduled,

@@ -58,6 +58,20 @@
  * ctx_len[r] counts the KV entries committed BEFORE the round; the round
  * appends gamma+1 entries at positions ctx_len[r] .. ctx_len[r]+gamma, and
  * query row i of the request sees keys [0, ctx_len[r] + i].
+ *
+ * Ragged rows (per-request draft depth).  The target verifies the anchor plus the
+ * proposal tokens of each request (Appendix G.2), and the draft depth is a knob of
+ * the draft side (the depth study runs 3, 4 and 5), so one batch may mix depths.
+ * Every call that takes a `q_indptr` (int64 [batch+1], q_indptr[0] = 0) then works
+ * on ragged row tensors: request r has gamma_r = q_indptr[r+1] - q_indptr[r] - 1
+ * proposals (0 <= gamma_r <= gamma, the `gamma` argument being the upper bound), its
+ * gamma_r + 1 query / new-token / target-probability rows start at row q_indptr[r]
+ * of tensors with q_indptr[batch] rows in all, and its gamma_r draft rows, draft
+ * tokens and accept uniforms start at q_indptr[r] - r (one fewer per request) of
+ * tensors with q_indptr[batch] - batch entries.  No padded row is read, computed or
+ * appended.  With q_indptr null every request has gamma proposals and the tensors
+ * have the padded shapes given at each call.  A depth outside [0, gamma] met on the
+ * device is skipped and reported by nsd_get_status as DEVICE_FAULT.
  */
 #ifndef NSD_H_
 #define NSD_H_
@@ -153,6 +167,9 @@ nsd_status nsd_destroy(nsd_ctx* ctx);
  *                             without it serves any round, but such a round cannot
  *                             overlap its first layer with its own copy (it waits for
  *                             the copy, then attends everybody) and cannot fuse_gather
+ *   h_q_indptr     [batch+1]  nullable; per-request draft depth (see "Ragged rows" below): request
+ *                             r brings h_q_indptr[r+1] - h_q_indptr[r] - 1 proposals, each depth in
+ *                             [0, gamma]; h_q_indptr[0] = 0.  Null: every request has gamma proposals
  *   chunk_blocks   0 = choose; else the split-KV chunk length in blocks (even, <= 256)
  * Errors: INVALID_ARG (null, negative length, short table), OUT_OF_RANGE
  * (batch > max_batch, gamma outside [1,max_gamma]), CAPACITY (table entries or
@@ -160,8 +177,8 @@ nsd_status nsd_destroy(nsd_ctx* ctx);
  * batch == 0 is a valid empty plan.
  */
 nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
-                           const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
-                           void* stream);
+                           const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, const int64_t* h_q_indptr,
+                           int32_t chunk_blocks, void* stream);
 
 /*
  * KV-state preparation (Section 3 "fragmented copies"; Section 5 / Appendix E.2:
@@ -182,6 +199,9 @@ nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int
  *   is_migrated nullable uint8 [batch]; append_subset: 0 = every request,
  *               1 = only requests with is_migrated == 0, 2 = only == 1
  *               (1 and 2 need is_migrated)
+ *   q_indptr    nullable device int64 [batch+1]: ragged rows; total_rows =
+ *               q_indptr[batch] as the host knows it (the rows of one layer of
+ *               k_new / v_new; ignored when q_indptr is null)
  * Destination and append blocks must be unique per request, else the result is
  * undefined (not checked).  Errors: INVALID_ARG, OUT_OF_RANGE (layers, gamma,
  * batch).  A bad block id on the device is skipped and reported by
@@ -191,7 +211,8 @@ nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
                           const int32_t* mig_src, const int32_t* mig_dst, int32_t batch, int32_t gamma,
                           const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices,
                           const void* k_new, const void* v_new, const uint8_t* is_migrated,
-                          int32_t append_subset, int32_t layer_begin, int32_t layer_count, void* stream);
+                          int32_t append_subset, int32_t layer_begin, int32_t layer_count, const int64_t* q_indptr,
+                          int64_t total_rows, void* stream);
 
 /*
  * Verification attention for one logical layer (Appendix G.2: the target
@@ -199,7 +220,8 @@ nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
  * sqrt(head_dim)) V, q head h reading kv head h / (num_q_heads/num_kv_heads)).
  * Uses the batch last given to nsd_verify_plan; ctx_len / kv_indptr must hold
  * the same values on the device.
- *   q    bf16 [batch*(gamma+1)][num_q_heads][head_dim]   (this layer's rows)
+ *   q    bf16 [batch*(gamma+1)][num_q_heads][head_dim]   (this layer's rows; ragged when the plan
+ *        was given h_q_indptr: [q_indptr[batch]] rows, request r's from row q_indptr[r])
  *   o    bf16 same shape (written for the requests of `subset`)
  *   lse  nullable fp32 [batch*(gamma+1)][num_q_heads], natural-log sum-exp
  *   subset  0 = all requests, 1 = resident only, 2 = reassigned only
@@ -223,13 +245,16 @@ nsd_status nsd_verify_attn(nsd_ctx* ctx, const void* kv_pool, const void* q, voi
  *   acc_len int32 [batch]             out_tok int32 [batch][gamma+1]: accepted
  *   drafts, then y, then -1 padding
  *   ctx_len / new_ctx_len  nullable pair: new_ctx_len[r] = ctx_len[r] + 1 + n
+ *   q_indptr  nullable device int64 [batch+1]: ragged rows -- p [rows][vocab], q [rows - batch][vocab],
+ *   draft_tok / u_acc [rows - batch], out_tok [rows], rows = q_indptr[batch]; a request without
+ *   proposals emits the token drawn from its one target row
  * Errors: INVALID_ARG, OUT_OF_RANGE (gamma, batch, vocab < 1).  A draft token
  * outside [0, vocab) counts as rejected and is reported as DEVICE_FAULT.
  */
 nsd_status nsd_spec_accept(nsd_ctx* ctx, const float* p, const float* q, const int32_t* draft_tok,
                            const float* u_acc, const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab,
                            const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len,
-                           void* stream);
+                           const int64_t* q_indptr, void* stream);
 
 /*
  * Acceptance straight from the target's logits: the step in front of nsd_spec_accept
@@ -267,7 +292,8 @@ nsd_status nsd_spec_accept_logits(nsd_ctx* ctx, const void* logits, int32_t logi
  * exp_indices names for the same position (entry index position / block_size, same
  * slot).  Rejected drafts stay behind.  acc_len is read on the device, so the call
  * can be enqueued right behind nsd_spec_accept / nsd_verify_round.
- *   acc_len      int32 [batch], each in [0, gamma] (else reported as DEVICE_FAULT)
+ *   acc_len      int32 [batch], each in [0, gamma] -- in [0, gamma_r] with q_indptr (nullable
+ *                device int64 [batch+1], ragged rows) -- else reported as DEVICE_FAULT
  *   exp_indptr / exp_indices   the export copy's table; entries that cannot hold
  *                a committed position are never read (may be -1)
  *   new_ctx_len  nullable int32 [batch]: ctx_len[r] + 1 + acc_len[r]
@@ -277,7 +303,7 @@ nsd_status nsd_spec_accept_logits(nsd_ctx* ctx, const void* logits, int32_t logi
 nsd_status nsd_kv_commit(nsd_ctx* ctx, void* kv_pool, int32_t batch, int32_t gamma, const int32_t* ctx_len,
                          const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
                          const int64_t* exp_indptr, const int32_t* exp_indices, int32_t* new_ctx_len,
-                         int32_t layer_begin, int32_t layer_count, void* stream);
+                         int32_t layer_begin, int32_t layer_count, const int64_t* q_indptr, void* stream);
 
 /* Per-round tensors of nsd_verify_round; every pointer on the device. */
 typedef struct {
@@ -305,6 +331,9 @@ typedef struct {
     int32_t* new_ctx_len;         /* nullable */
     int32_t fuse_gather;          /* 0 = side-stream gather (default), 1 = gather-through attention */
     int32_t reserved;
+    const int64_t* q_indptr;      /* nullable: ragged rows (the plan must have been given the same depths);
+                                     every row tensor above then has q_indptr[batch] rows per layer,
+                                     q_draft / draft_tok / u_acc q_indptr[batch] - batch entries */
 } nsd_round_args;
 
 /*

@@ -57,6 +57,7 @@ class RoundArgs(ctypes.Structure):
         ("kv_indices", _vp), ("is_migrated", _vp), ("k_new", _vp), ("v_new", _vp), ("q", _vp), ("o", _vp),
         ("p", _vp), ("q_draft", _vp), ("draft_tok", _vp), ("u_acc", _vp), ("u_smp", _vp), ("acc_len", _vp),
         ("out_tok", _vp), ("new_ctx_len", _vp), ("fuse_gather", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("q_indptr", _vp),
     ]
 
 
@@ -89,15 +90,15 @@ def load_library():
     lib.nsd_destroy.restype = i32
     lib.nsd_destroy.argtypes = [_vp]
     lib.nsd_verify_plan.restype = i32
-    lib.nsd_verify_plan.argtypes = [_vp, i32, i32, _vp, _vp, _vp, i32, _vp]
+    lib.nsd_verify_plan.argtypes = [_vp, i32, i32, _vp, _vp, _vp, _vp, i32, _vp]
     lib.nsd_kv_prepare.restype = i32
-    lib.nsd_kv_prepare.argtypes = [_vp, _vp, i64, _vp, _vp, i32, i32, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp]
+    lib.nsd_kv_prepare.argtypes = [_vp, _vp, i64, _vp, _vp, i32, i32, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp, i64, _vp]
     lib.nsd_kv_commit.restype = i32
-    lib.nsd_kv_commit.argtypes = [_vp, _vp, i32, i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, _vp]
+    lib.nsd_kv_commit.argtypes = [_vp, _vp, i32, i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, i32, i32, _vp, _vp]
     lib.nsd_verify_attn.restype = i32
     lib.nsd_verify_attn.argtypes = [_vp, _vp, _vp, _vp, _vp, i32, i32, _vp, _vp, _vp, i32, i32, _vp]
     lib.nsd_spec_accept.restype = i32
-    lib.nsd_spec_accept.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp, _vp, _vp, _vp, _vp]
+    lib.nsd_spec_accept.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, i32, i32, i32, _vp, _vp, _vp, _vp, _vp, _vp]
     lib.nsd_spec_accept_logits.restype = i32
     lib.nsd_spec_accept_logits.argtypes = [_vp, _vp, i32, ctypes.c_float, _vp, _vp, _vp, _vp, i32, i32, i32, _vp, _vp, _vp, _vp, _vp, _vp]
     lib.nsd_verify_round.restype = i32
@@ -221,29 +222,30 @@ class VerifyContext:
             pass
 
     # -- the C ABI, one method per entry point
-    def nsd_verify_plan(self, h_ctx_len, h_kv_indptr, h_is_migrated, gamma, chunk_blocks=0, stream=None):
+    def nsd_verify_plan(self, h_ctx_len, h_kv_indptr, h_is_migrated, gamma, chunk_blocks=0, stream=None, h_q_indptr=None):
         batch = len(h_ctx_len)
         self._check(self.lib.nsd_verify_plan(self._h, batch, gamma, _ptr(h_ctx_len), _ptr(h_kv_indptr),
-                                             _ptr(h_is_migrated), chunk_blocks, _stream_handle(stream)),
+                                             _ptr(h_is_migrated), _ptr(h_q_indptr), chunk_blocks, _stream_handle(stream)),
                     "nsd_verify_plan")
 
     def nsd_kv_prepare(self, kv_pool, n_mig_blocks, mig_src, mig_dst, batch, gamma, ctx_len, kv_indptr, kv_indices,
-                       k_new, v_new, is_migrated=None, append_subset=0, layer_begin=0, layer_count=None, stream=None):
+                       k_new, v_new, is_migrated=None, append_subset=0, layer_begin=0, layer_count=None, stream=None,
+                       q_indptr=None, total_rows=0):
         if layer_count is None:
             layer_count = self.cfg.num_layers - layer_begin
         self._check(self.lib.nsd_kv_prepare(self._h, _ptr(kv_pool), n_mig_blocks, _ptr(mig_src), _ptr(mig_dst), batch,
                                             gamma, _ptr(ctx_len), _ptr(kv_indptr), _ptr(kv_indices), _ptr(k_new),
                                             _ptr(v_new), _ptr(is_migrated), append_subset, layer_begin, layer_count,
-                                            _stream_handle(stream)), "nsd_kv_prepare")
+                                            _ptr(q_indptr), int(total_rows), _stream_handle(stream)), "nsd_kv_prepare")
 
     def nsd_kv_commit(self, kv_pool, batch, gamma, ctx_len, acc_len, kv_indptr, kv_indices, exp_indptr, exp_indices,
-                      new_ctx_len=None, layer_begin=0, layer_count=None, stream=None):
+                      new_ctx_len=None, layer_begin=0, layer_count=None, stream=None, q_indptr=None):
         if layer_count is None:
             layer_count = self.cfg.num_layers - layer_begin
         self._check(self.lib.nsd_kv_commit(self._h, _ptr(kv_pool), batch, gamma, _ptr(ctx_len), _ptr(acc_len),
                                            _ptr(kv_indptr), _ptr(kv_indices), _ptr(exp_indptr), _ptr(exp_indices),
-                                           _ptr(new_ctx_len), layer_begin, layer_count, _stream_handle(stream)),
-                    "nsd_kv_commit")
+                                           _ptr(new_ctx_len), layer_begin, layer_count, _ptr(q_indptr),
+                                           _stream_handle(stream)), "nsd_kv_commit")
 
     def nsd_verify_attn(self, kv_pool, q, o, lse, batch, gamma, ctx_len, kv_indptr, kv_indices, layer=0, subset=0,
                         stream=None):
@@ -252,10 +254,10 @@ class VerifyContext:
                                              _stream_handle(stream)), "nsd_verify_attn")
 
     def nsd_spec_accept(self, p, q, draft_tok, u_acc, u_smp, batch, gamma, vocab, ctx_len, acc_len, out_tok,
-                        new_ctx_len=None, stream=None):
+                        new_ctx_len=None, stream=None, q_indptr=None):
         self._check(self.lib.nsd_spec_accept(self._h, _ptr(p), _ptr(q), _ptr(draft_tok), _ptr(u_acc), _ptr(u_smp),
                                              batch, gamma, vocab, _ptr(ctx_len), _ptr(acc_len), _ptr(out_tok),
-                                             _ptr(new_ctx_len), _stream_handle(stream)), "nsd_spec_accept")
+                                             _ptr(new_ctx_len), _ptr(q_indptr), _stream_handle(stream)), "nsd_spec_accept")
 
     def nsd_spec_accept_logits(self, logits, logits_dtype, temperature, q, draft_tok, u_acc, u_smp, batch, gamma, vocab,
                                gamma_r, ctx_len, acc_len, out_tok, new_ctx_len=None, stream=None):

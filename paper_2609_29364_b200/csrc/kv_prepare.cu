@@ -129,7 +129,7 @@ gather_blocks_bulk_kernel(uint16_t* __restrict__ slab, int64_t n_pairs, const in
 // One warp per (row, K|V): copies the Hkv head vectors of one new token into its slot.
 __global__ void __launch_bounds__(256)
 append_tokens_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32_t gamma,
-                     const int32_t* __restrict__ ctx_len, const int64_t* __restrict__ kv_indptr,
+                     const int64_t* __restrict__ q_indptr, const int32_t* __restrict__ ctx_len, const int64_t* __restrict__ kv_indptr,
                      const int32_t* __restrict__ kv_indices, const uint16_t* __restrict__ k_new,
                      const uint16_t* __restrict__ v_new, const uint8_t* __restrict__ is_migrated, int32_t subset,
                      int32_t* __restrict__ status) {
@@ -138,10 +138,22 @@ append_tokens_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32
     const int64_t n_rows = (int64_t)batch * (gamma + 1);
     if (warp >= 2 * n_rows) return;
     const int kv = (int)(warp & 1);
-    const int64_t row = warp >> 1;
+    int64_t row = warp >> 1;                                        // (request, token) over the padded grid batch x (gamma + 1)
     const int r = (int)(row / (gamma + 1));
     const int t = (int)(row - (int64_t)r * (gamma + 1));
     if (subset != 0 && (int)(is_migrated[r] != 0) != (subset == 2)) return;
+    if (q_indptr) {                                                 // ragged rows: the request has its own depth and row offset
+        const int64_t r0 = q_indptr[r], n = q_indptr[r + 1] - r0;
+        if (n < 1 || n > gamma + 1) {
+            if (lane == 0 && t == 0 && kv == 0) {
+                atomicOr(status, STATUS_BAD_TOKEN);
+                atomicCAS(status + 1, 0, r + 1);
+            }
+            return;
+        }
+        if (t >= n) return;
+        row = r0 + t;
+    }
     const int64_t pos = (int64_t)ctx_len[r] + t;
     const int64_t entry = kv_indptr[r] + pos / sh.bs;
     const int slot = (int)(pos % sh.bs);
@@ -170,7 +182,7 @@ append_tokens_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32
 // needs no host round trip after the acceptance kernel.
 __global__ void __launch_bounds__(256)
 commit_suffix_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32_t gamma,
-                     const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ acc_len,
+                     const int64_t* __restrict__ q_indptr, const int32_t* __restrict__ ctx_len, const int32_t* __restrict__ acc_len,
                      const int64_t* __restrict__ kv_indptr, const int32_t* __restrict__ kv_indices,
                      const int64_t* __restrict__ exp_indptr, const int32_t* __restrict__ exp_indices,
                      int32_t* __restrict__ new_ctx_len, int32_t* __restrict__ status) {
@@ -183,7 +195,9 @@ commit_suffix_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32
     const int r = (int)(row / (gamma + 1));
     const int t = (int)(row - (int64_t)r * (gamma + 1));
     const int acc = acc_len[r];
-    if ((uint32_t)acc > (uint32_t)gamma) {
+    // at most the drafts the request had: gamma, or its own depth when the rows are ragged
+    const int depth = q_indptr ? (int)min((int64_t)gamma, q_indptr[r + 1] - q_indptr[r] - 1) : gamma;
+    if (acc < 0 || acc > depth) {
         if (lane == 0 && t == 0 && kv == 0) {
             atomicOr(status, STATUS_BAD_TOKEN);
             atomicCAS(status + 1, 0, r + 1);
@@ -239,26 +253,26 @@ cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const
     return cudaGetLastError();
 }
 
-cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int32_t* ctx_len,
-                          const int64_t* kv_indptr, const int32_t* kv_indices, const uint16_t* k_new,
+cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int64_t* q_indptr,
+                          const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices, const uint16_t* k_new,
                           const uint16_t* v_new, const uint8_t* is_migrated, int32_t subset, int32_t* status,
                           cudaStream_t stream) {
     const int64_t warps = 2LL * batch * (gamma + 1);
     if (warps <= 0) return cudaSuccess;
     const int grid = (int)((warps * 32 + 255) / 256);
-    append_tokens_kernel<<<grid, 256, 0, stream>>>(slab, s, batch, gamma, ctx_len, kv_indptr, kv_indices, k_new, v_new,
+    append_tokens_kernel<<<grid, 256, 0, stream>>>(slab, s, batch, gamma, q_indptr, ctx_len, kv_indptr, kv_indices, k_new, v_new,
                                                    is_migrated, subset, status);
     return cudaGetLastError();
 }
 
-cudaError_t launch_commit(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int32_t* ctx_len,
-                          const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
+cudaError_t launch_commit(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int64_t* q_indptr,
+                          const int32_t* ctx_len, const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
                           const int64_t* exp_indptr, const int32_t* exp_indices, int32_t* new_ctx_len, int32_t* status,
                           cudaStream_t stream) {
     const int64_t warps = 2LL * batch * (gamma + 1);
     if (warps <= 0) return cudaSuccess;
     const int grid = (int)((warps * 32 + 255) / 256);
-    commit_suffix_kernel<<<grid, 256, 0, stream>>>(slab, s, batch, gamma, ctx_len, acc_len, kv_indptr, kv_indices, exp_indptr,
+    commit_suffix_kernel<<<grid, 256, 0, stream>>>(slab, s, batch, gamma, q_indptr, ctx_len, acc_len, kv_indptr, kv_indices, exp_indptr,
                                                    exp_indices, new_ctx_len, status);
     return cudaGetLastError();
 }

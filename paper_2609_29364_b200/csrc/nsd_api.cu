@@ -13,6 +13,8 @@
 
 using namespace nsd;
 
+constexpr int kAttnClasses = 6;
+
 struct nsd_ctx {
     nsd_config cfg;
     Shape shape;
@@ -36,6 +38,13 @@ struct nsd_ctx {
     bool planned;
     int32_t plan_batch, plan_gamma;
     int32_t n_all, n_res, n_mig_items;
+    // Items are grouped by row-tile class (how many 8-row tiles their stacked query rows need: the kernel is instantiated
+    // per class) and, inside a class, ordered longest first.  cls_*[c] .. cls_*[c+1] = the items of class c in the list of
+    // all items, in the resident part and in the reassigned part of the split list.
+    int32_t cls_all[kAttnClasses + 1], cls_res[kAttnClasses + 1], cls_mig[kAttnClasses + 1];
+    int64_t plan_rows;         // query rows of the planned batch: batch * (gamma + 1), or the ragged total
+    bool plan_ragged;          // the plan was given per-request depths (h_q_indptr)
+    int32_t plan_m_stride;     // rows per split-KV partial slot
     int32_t plan_split_slots;  // partial slots the plan uses (0 = no request is split)
     int64_t plan_src_blocks;   // source blocks of the planned batch's reassigned requests
     bool plan_has_mig;         // the plan was given is_migrated (its resident / reassigned item lists are meaningful)
@@ -61,6 +70,16 @@ struct nsd_ctx {
 };
 
 namespace {
+
+// Row-tile classes of the attention kernel: (warps, 8-row tiles per warp) = 1x1, 1x2, 1x3, 2x2, 2x3, 3x3.
+int attn_class_of(int m_rows) {
+    const int nt8 = (m_rows + 7) / 8;
+    return nt8 <= 3 ? nt8 - 1 : (nt8 == 4 ? 3 : (nt8 <= 6 ? 4 : 5));
+}
+int attn_class_rows(int cls) {
+    static const int rows[kAttnClasses] = {8, 16, 24, 32, 48, 64};
+    return rows[cls];
+}
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -273,22 +292,22 @@ nsd_status nsd_destroy(nsd_ctx* ctx) {
 }
 
 static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
-                                   const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
-                                   void* stream);
+                                   const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, const int64_t* h_q_indptr,
+                                   int32_t chunk_blocks, void* stream);
 
 nsd_status nsd_verify_plan(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
-                           const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
-                           void* stream) {
+                           const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, const int64_t* h_q_indptr,
+                           int32_t chunk_blocks, void* stream) {
     try {
-        return verify_plan_impl(ctx, batch, gamma, h_ctx_len, h_kv_indptr, h_is_migrated, chunk_blocks, stream);
+        return verify_plan_impl(ctx, batch, gamma, h_ctx_len, h_kv_indptr, h_is_migrated, h_q_indptr, chunk_blocks, stream);
     } catch (...) {                        // the host work list could not be allocated: nothing crosses the C boundary
         return NSD_ERR_CAPACITY;
     }
 }
 
 static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* h_ctx_len,
-                                   const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, int32_t chunk_blocks,
-                                   void* stream) {
+                                   const int64_t* h_kv_indptr, const uint8_t* h_is_migrated, const int64_t* h_q_indptr,
+                                   int32_t chunk_blocks, void* stream) {
     if (!ctx) return NSD_ERR_INVALID_ARG;
     if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
     if (chunk_blocks < 0 || (chunk_blocks & 1) || chunk_blocks > 256) return NSD_ERR_INVALID_ARG;
@@ -296,11 +315,19 @@ static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, c
     const int bs = ctx->cfg.block_size;
     const int Hkv = ctx->cfg.num_kv_heads;
     // ---- validate lengths and tables
-    std::vector<int32_t> nblk(batch);
+    std::vector<int32_t> nblk(batch), depth(batch, gamma);
+    std::vector<int64_t> row0(batch + 1, 0);
     int64_t total_blocks = 0;
+    if (batch > 0 && h_q_indptr && h_q_indptr[0] != 0) return NSD_ERR_INVALID_ARG;
     for (int r = 0; r < batch; ++r) {
+        if (h_q_indptr) {                                                   // per-request draft depth, rows ragged
+            const int64_t n = h_q_indptr[r + 1] - h_q_indptr[r];
+            if (n < 1 || n > gamma + 1) return NSD_ERR_OUT_OF_RANGE;
+            depth[r] = (int32_t)n - 1;
+        }
+        row0[r + 1] = row0[r] + depth[r] + 1;
         if (h_ctx_len[r] < 0 || h_kv_indptr[r] < 0 || h_kv_indptr[r + 1] < h_kv_indptr[r]) return NSD_ERR_INVALID_ARG;
-        const int64_t need = ((int64_t)h_ctx_len[r] + gamma + 1 + bs - 1) / bs;
+        const int64_t need = ((int64_t)h_ctx_len[r] + depth[r] + 1 + bs - 1) / bs;
         if (h_kv_indptr[r + 1] - h_kv_indptr[r] < need) return NSD_ERR_INVALID_ARG;
         if (need > INT32_MAX / 2) return NSD_ERR_OUT_OF_RANGE;
         nblk[r] = (int32_t)need;
@@ -308,6 +335,7 @@ static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, c
     }
     if (batch > 0 && h_kv_indptr[batch] > ctx->cfg.max_table_entries) return NSD_ERR_CAPACITY;
     if (batch > 0 && h_kv_indptr[batch] > INT32_MAX) return NSD_ERR_CAPACITY;      // items carry table offsets as int32
+    if (row0[batch] > INT32_MAX / 2) return NSD_ERR_CAPACITY;                       // ... and row offsets
 
     // ---- chunk length: split only as far as it takes to give every resident CTA slot of the machine one item.
     //      Measured: a split costs a partial store, a counter and a merge (several microseconds at the end of a
@@ -344,7 +372,8 @@ static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, c
         cb = std::min(256, cb * 2);
     }
     // ---- items
-    struct Tmp { AttnItem it; int mig; };
+    const int G = ctx->cfg.num_q_heads / ctx->cfg.num_kv_heads;
+    struct Tmp { AttnItem it; int mig; int cls; };
     std::vector<Tmp> items;
     int32_t slot = 0;
     int64_t src_next = 0;                                                // running offset into the gather's pair list
@@ -369,12 +398,15 @@ static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, c
             it.src_off = (int32_t)src_off;
             it.ctx = h_ctx_len[r];
             it.tbl_off = (int32_t)h_kv_indptr[r];
-            items.push_back({it, h_is_migrated ? (h_is_migrated[r] != 0) : 0});
+            it.gamma = depth[r];
+            it.row0 = (int32_t)row0[r];
+            items.push_back({it, h_is_migrated ? (h_is_migrated[r] != 0) : 0, attn_class_of(G * (depth[r] + 1))});
         }
         if (n_eff > 1) slot += n_eff;
     }
     if ((int64_t)items.size() > ctx->max_items || slot > ctx->part_slots) return NSD_ERR_CAPACITY;
     auto longer = [](const Tmp& a, const Tmp& b) {
+        if (a.cls != b.cls) return a.cls > b.cls;                           // the widest row tiles first
         const int la = a.it.blk_end - a.it.blk_begin, lb = b.it.blk_end - b.it.blk_begin;
         if (la != lb) return la > lb;
         if (a.it.req != b.it.req) return a.it.req < b.it.req;
@@ -397,6 +429,26 @@ static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, c
         NSD_CUDA(ctx, cudaMemcpyAsync(ctx->d_items_split, split, (size_t)n_all * sizeof(AttnItem), cudaMemcpyHostToDevice, st));
     }
     NSD_CUDA(ctx, cudaEventRecord(ctx->ev_plan_free, st));
+    {
+        // class boundaries of the three lists (classes run from the widest to the narrowest)
+        auto bounds = [&](int32_t* off, int mig_filter) {
+            int32_t count[kAttnClasses] = {0};
+            for (const Tmp& t : items)
+                if (mig_filter < 0 || t.mig == mig_filter) count[t.cls]++;
+            int32_t run = 0;
+            for (int c = kAttnClasses - 1; c >= 0; --c) {                 // position c' = kAttnClasses - 1 - c in list order
+                off[kAttnClasses - 1 - c] = run;
+                run += count[c];
+            }
+            off[kAttnClasses] = run;
+        };
+        bounds(ctx->cls_all, -1);
+        bounds(ctx->cls_res, 0);
+        bounds(ctx->cls_mig, 1);
+    }
+    ctx->plan_rows = row0[batch];
+    ctx->plan_ragged = h_q_indptr != nullptr;
+    ctx->plan_m_stride = G * (gamma + 1);
     ctx->planned = true;
     ctx->plan_batch = batch;
     ctx->plan_gamma = gamma;
@@ -413,7 +465,8 @@ nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
                           const int32_t* mig_src, const int32_t* mig_dst, int32_t batch, int32_t gamma,
                           const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices,
                           const void* k_new, const void* v_new, const uint8_t* is_migrated,
-                          int32_t append_subset, int32_t layer_begin, int32_t layer_count, void* stream) {
+                          int32_t append_subset, int32_t layer_begin, int32_t layer_count, const int64_t* q_indptr,
+                          int64_t total_rows, void* stream) {
     if (!ctx || !kv_pool) return NSD_ERR_INVALID_ARG;
     if (n_mig_blocks < 0 || layer_count < 0) return NSD_ERR_INVALID_ARG;
     if (batch < 0 || batch > ctx->cfg.max_batch) return NSD_ERR_OUT_OF_RANGE;
@@ -427,7 +480,8 @@ nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
     if (n_mig_blocks > 0 && (!mig_src || !mig_dst)) return NSD_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t n_pairs = n_mig_blocks;
-    const int64_t layer_rows = (int64_t)batch * (gamma + 1) * ctx->cfg.num_kv_heads * ctx->cfg.head_dim;
+    if (q_indptr && (total_rows < batch || total_rows > (int64_t)batch * (gamma + 1))) return NSD_ERR_INVALID_ARG;
+    const int64_t layer_rows = (q_indptr ? total_rows : (int64_t)batch * (gamma + 1)) * ctx->cfg.num_kv_heads * ctx->cfg.head_dim;
     for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
         uint16_t* slab = slab_ptr(ctx, kv_pool, l);
         if (n_pairs > 0) {
@@ -435,7 +489,7 @@ nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
             ctx->launches++;
         }
         if (do_append && batch > 0) {
-            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, ctx_len, kv_indptr, kv_indices,
+            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, q_indptr, ctx_len, kv_indptr, kv_indices,
                                         static_cast<const uint16_t*>(k_new) + (int64_t)l * layer_rows,
                                         static_cast<const uint16_t*>(v_new) + (int64_t)l * layer_rows, is_migrated,
                                         append_subset, ctx->d_status, st));
@@ -448,7 +502,7 @@ nsd_status nsd_kv_prepare(nsd_ctx* ctx, void* kv_pool, int64_t n_mig_blocks,
 nsd_status nsd_kv_commit(nsd_ctx* ctx, void* kv_pool, int32_t batch, int32_t gamma, const int32_t* ctx_len,
                          const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
                          const int64_t* exp_indptr, const int32_t* exp_indices, int32_t* new_ctx_len,
-                         int32_t layer_begin, int32_t layer_count, void* stream) {
+                         int32_t layer_begin, int32_t layer_count, const int64_t* q_indptr, void* stream) {
     if (!ctx) return NSD_ERR_INVALID_ARG;
     if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma) return NSD_ERR_OUT_OF_RANGE;
     if (layer_count < 0) return NSD_ERR_INVALID_ARG;
@@ -457,7 +511,7 @@ nsd_status nsd_kv_commit(nsd_ctx* ctx, void* kv_pool, int32_t batch, int32_t gam
     if (!kv_pool || !ctx_len || !acc_len || !kv_indptr || !kv_indices || !exp_indptr || !exp_indices) return NSD_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     for (int l = layer_begin; l < layer_begin + layer_count; ++l) {
-        NSD_CUDA(ctx, launch_commit(ctx->shape, slab_ptr(ctx, kv_pool, l), batch, gamma, ctx_len, acc_len, kv_indptr,
+        NSD_CUDA(ctx, launch_commit(ctx->shape, slab_ptr(ctx, kv_pool, l), batch, gamma, q_indptr, ctx_len, acc_len, kv_indptr,
                                     kv_indices, exp_indptr, exp_indices, l == layer_begin ? new_ctx_len : nullptr,
                                     ctx->d_status, st));
         ctx->launches++;
@@ -496,13 +550,12 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
     a.part_ml = ctx->d_part_ml;
     a.counters = ctx->d_counters;
     a.status = ctx->d_status;
-    a.m_rows = (ctx->cfg.num_q_heads / ctx->cfg.num_kv_heads) * (gamma + 1);
-    if (subset == 0) { a.items = ctx->d_items_all; a.n_items = ctx->n_all; }
-    else if (subset == 1) { a.items = ctx->d_items_split; a.n_items = ctx->n_res; }
-    else { a.items = ctx->d_items_split + ctx->n_res; a.n_items = ctx->n_mig_items; }
-    if (a.n_items == 0) return NSD_OK;
+    a.m_stride = ctx->plan_m_stride;
     a.wait_budget = ctx->wait_budget;
     a.any_split = ctx->plan_split_slots > 0;
+    const AttnItem* base = subset == 0 ? ctx->d_items_all : (subset == 1 ? ctx->d_items_split : ctx->d_items_split + ctx->n_res);
+    const int32_t* cls = subset == 0 ? ctx->cls_all : (subset == 1 ? ctx->cls_res : ctx->cls_mig);
+    if (cls[kAttnClasses] == 0) return NSD_OK;
     if ((ctx->attn_feed_tma || ctx->attn_tcgen05) && !fuse && ctx->cfg.head_dim == 128) {
         const int slab = layer % ctx->cfg.num_slabs;
         if (ctx->tmap_slab[slab] != a.pool_slab) {
@@ -518,14 +571,22 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
             }
         }
         a.tma_feed = ctx->attn_feed_tma;
-        if (ctx->attn_tcgen05 && attn_umma_supported(a) && (ctx->attn_tcgen05 == 2 || attn_umma_preferred(a))) {
+    }
+    // one launch per row-tile class present (a batch of one draft depth has one), widest first
+    for (int pos = 0; pos < kAttnClasses; ++pos) {
+        const int n = cls[pos + 1] - cls[pos];
+        if (n == 0) continue;
+        a.items = base + cls[pos];
+        a.n_items = n;
+        a.m_rows = std::min(attn_class_rows(kAttnClasses - 1 - pos), ctx->plan_m_stride);
+        if (a.tmap_valid && ctx->attn_tcgen05 && attn_umma_supported(a) && (ctx->attn_tcgen05 == 2 || attn_umma_preferred(a))) {
             NSD_CUDA(ctx, launch_attn_umma(a, st, ctx->n_sms));
             ctx->launches += a.any_split ? 2 : 1;                            // the engine's merge kernel follows when a request is split
-            return NSD_OK;
+            continue;
         }
+        NSD_CUDA(ctx, launch_attn(a, st));
+        ctx->launches++;
     }
-    NSD_CUDA(ctx, launch_attn(a, st));
-    ctx->launches++;
     return NSD_OK;
 }
 }  // namespace
@@ -547,13 +608,13 @@ nsd_status nsd_verify_attn(nsd_ctx* ctx, const void* kv_pool, const void* q, voi
 nsd_status nsd_spec_accept(nsd_ctx* ctx, const float* p, const float* q, const int32_t* draft_tok,
                            const float* u_acc, const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab,
                            const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len,
-                           void* stream) {
+                           const int64_t* q_indptr, void* stream) {
     if (!ctx) return NSD_ERR_INVALID_ARG;
     if (batch < 0 || batch > ctx->cfg.max_batch || gamma < 1 || gamma > ctx->cfg.max_gamma || vocab < 1) return NSD_ERR_OUT_OF_RANGE;
     if (batch == 0) return NSD_OK;
     if (!p || !q || !draft_tok || !u_acc || !u_smp || !acc_len || !out_tok) return NSD_ERR_INVALID_ARG;
     if ((new_ctx_len != nullptr) && !ctx_len) return NSD_ERR_INVALID_ARG;
-    NSD_CUDA(ctx, launch_accept(p, q, draft_tok, u_acc, u_smp, batch, gamma, vocab, ctx_len, acc_len, out_tok,
+    NSD_CUDA(ctx, launch_accept(p, q, draft_tok, u_acc, u_smp, batch, gamma, vocab, q_indptr, ctx_len, acc_len, out_tok,
                                 new_ctx_len, ctx->d_status, ctx->accept_split, static_cast<cudaStream_t>(stream)));
     ctx->launches++;
     return NSD_OK;
@@ -610,8 +671,10 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int L = ctx->cfg.num_layers, S = ctx->cfg.num_slabs;
     const int Hq = ctx->cfg.num_q_heads, Hkv = ctx->cfg.num_kv_heads, D = ctx->cfg.head_dim;
-    const int64_t rows = (int64_t)batch * (gamma + 1);
+    if ((a->q_indptr != nullptr) != ctx->plan_ragged) return NSD_ERR_INVALID_ARG;   // the plan fixed the rows' layout
+    const int64_t rows = ctx->plan_rows;
     const int64_t kv_layer = rows * Hkv * D, q_layer = rows * Hq * D;
+    const int64_t* qi = a->q_indptr;
     const uint16_t* k_new = static_cast<const uint16_t*>(a->k_new);
     const uint16_t* v_new = static_cast<const uint16_t*>(a->v_new);
     const uint16_t* q = static_cast<const uint16_t*>(a->q);
@@ -651,18 +714,18 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
             nsd_status s;
             if (l == 0 && split_first) {
                 // nothing to hide the first copy behind but the first layer itself: its resident requests go first
-                NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, k_new, v_new,
+                NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices, k_new, v_new,
                                             a->is_migrated, 1, ctx->d_status, st));
                 s = attn_enqueue(ctx, a->kv_pool, q, o, nullptr, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, 0, 1, st);
                 if (s != NSD_OK) return s;
                 NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_prep[0], 0));
-                NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, k_new, v_new,
+                NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices, k_new, v_new,
                                             a->is_migrated, 2, ctx->d_status, st));
                 s = attn_enqueue(ctx, a->kv_pool, q, o, nullptr, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, 0, 2, st);
                 ctx->launches += 2;
             } else {
                 NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_prep[l], 0));
-                NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
+                NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices,
                                             k_new + l * kv_layer, v_new + l * kv_layer, nullptr, 0, ctx->d_status, st));
                 s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
                                  a->kv_indptr, a->kv_indices, l, 0, st);
@@ -673,7 +736,7 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
         } else if (fused) {
             // gather-through: only the resident requests are appended by the copy kernels; attention itself
             // moves the reassigned requests' blocks and new tokens while it streams them
-            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
+            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices,
                                         k_new + l * kv_layer, v_new + l * kv_layer, a->is_migrated, 1, ctx->d_status, st));
             ctx->launches++;
             const FuseArgs f{a->mig_src, k_new + l * kv_layer, v_new + l * kv_layer};
@@ -681,7 +744,7 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
                                         a->kv_indptr, a->kv_indices, l, 0, st, &f);
             if (s != NSD_OK) return s;
         } else {
-            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, a->ctx_len, a->kv_indptr, a->kv_indices,
+            NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices,
                                         k_new + l * kv_layer, v_new + l * kv_layer, nullptr, 0, ctx->d_status, st));
             ctx->launches++;
             nsd_status s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
@@ -699,7 +762,7 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
         NSD_CUDA(ctx, cudaEventRecord(ctx->ev_down_done, ctx->down));
         NSD_CUDA(ctx, cudaStreamWaitEvent(st, hook->inputs_ready, 0));
     }
-    NSD_CUDA(ctx, launch_accept(a->p, a->q_draft, a->draft_tok, a->u_acc, a->u_smp, batch, gamma, ctx->cfg.vocab_size,
+    NSD_CUDA(ctx, launch_accept(a->p, a->q_draft, a->draft_tok, a->u_acc, a->u_smp, batch, gamma, ctx->cfg.vocab_size, qi,
                                 a->ctx_len, a->acc_len, a->out_tok, a->new_ctx_len, ctx->d_status, ctx->accept_split, st));
     ctx->launches++;
     if (hook) NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down_done, 0));      // the caller's stream covers the read-back
@@ -718,7 +781,11 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
     if (batch == 0) return NSD_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int L = ctx->cfg.num_layers, Hq = ctx->cfg.num_q_heads, Hkv = ctx->cfg.num_kv_heads, D = ctx->cfg.head_dim;
-    const int64_t V = ctx->cfg.vocab_size, rows = (int64_t)batch * (gamma + 1);
+    if ((h->q_indptr != nullptr) != (d->q_indptr != nullptr)) return NSD_ERR_INVALID_ARG;
+    // ragged rows: the host copy of q_indptr gives the totals (target rows; one draft row fewer per request)
+    const int64_t V = ctx->cfg.vocab_size, rows = h->q_indptr ? h->q_indptr[batch] : (int64_t)batch * (gamma + 1);
+    if (rows < batch || rows > (int64_t)batch * (gamma + 1)) return NSD_ERR_INVALID_ARG;
+    const int64_t drafts = rows - batch;
     int64_t up = 0, down = 0;
     struct Copy { const void* src; const void* dst; int64_t bytes; };
     // Everything goes up on the copy stream in the order it is needed: the tables, then layer by layer the new K / V
@@ -732,12 +799,13 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
         {h->is_migrated, d->is_migrated, h->is_migrated ? batch * 1LL : 0},
         {h->mig_src, d->mig_src, h->n_mig_blocks * 4},
         {h->mig_dst, d->mig_dst, h->n_mig_blocks * 4},
+        {h->q_indptr, d->q_indptr, h->q_indptr ? (batch + 1) * 8LL : 0},
     };
     const Copy accept_in[] = {
-        {h->p, d->p, (int64_t)batch * (gamma + 1) * V * 4},
-        {h->q_draft, d->q_draft, (int64_t)batch * gamma * V * 4},
-        {h->draft_tok, d->draft_tok, (int64_t)batch * gamma * 4},
-        {h->u_acc, d->u_acc, (int64_t)batch * gamma * 4},
+        {h->p, d->p, rows * V * 4},
+        {h->q_draft, d->q_draft, drafts * V * 4},
+        {h->draft_tok, d->draft_tok, drafts * 4},
+        {h->u_acc, d->u_acc, drafts * 4},
         {h->u_smp, d->u_smp, batch * 4LL},
     };
     for (const Copy& c : tables)
@@ -746,7 +814,7 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
         if (c.bytes != 0 && (!c.src || !c.dst)) return NSD_ERR_INVALID_ARG;
     if (!h->k_new || !d->k_new || !h->v_new || !d->v_new || !h->q || !d->q) return NSD_ERR_INVALID_ARG;
     if (!h->o || !d->o || !h->acc_len || !d->acc_len || !h->out_tok || !d->out_tok) return NSD_ERR_INVALID_ARG;
-    nsd_status s = nsd_verify_plan(ctx, batch, gamma, h->ctx_len, h->kv_indptr, h->is_migrated, 0, stream);
+    nsd_status s = nsd_verify_plan(ctx, batch, gamma, h->ctx_len, h->kv_indptr, h->is_migrated, h->q_indptr, 0, stream);
     if (s != NSD_OK) return s;
     NSD_CUDA(ctx, cudaEventRecord(ctx->ev_copy_go, st));          // the device buffers are free once prior work is done
     NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->copy, ctx->ev_copy_go, 0));

@@ -20,7 +20,9 @@ struct __align__(16) AttnItem {
     int32_t src_off;     // first entry of the request's source blocks in the gather list, -1 = resident
     int32_t ctx;         // the request's context length when the plan was made (saves the kernels a dependent load)
     int32_t tbl_off;     // kv_indptr[req] when the plan was made (same); -1 = read kv_indptr[req] on the device
-    int32_t pad[3];
+    int32_t gamma;       // the request's draft depth: it has gamma + 1 query rows
+    int32_t row0;        // its first row in the row tensors (q, o, k_new, v_new): req * (gamma + 1), or the ragged offset
+    int32_t pad;
 };
 static_assert(sizeof(AttnItem) == 48, "AttnItem is read as three 16-byte words");
 
@@ -57,7 +59,8 @@ struct AttnLaunch {
     float* part_ml;              // [slot][Hkv][M][2]
     int32_t* counters;           // [max_batch][Hkv], zero between launches
     int32_t* status;
-    int32_t m_rows;              // (Hq/Hkv) * (gamma+1)
+    int32_t m_rows;              // stacked query rows the launch is shaped for: every item has (Hq/Hkv) * (item.gamma+1) <= m_rows
+    int32_t m_stride;            // rows per split-KV partial slot (the plan's largest m_rows)
     int32_t tmap_valid;          // tmap describes pool_slab
     int32_t tma_feed;            // mma.sync kernel: fetch K/V tiles with tensor copies where the shape allows
     uint32_t wait_budget;        // polls per bounded barrier wait, 0 = the kernel's default
@@ -71,12 +74,13 @@ struct AttnLaunch {
 // barrier expects and never receives (0 in production).
 cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const int32_t* src, const int32_t* dst,
                           int32_t* status, int n_sms, uint32_t wait_budget, uint32_t starve_bytes, cudaStream_t stream);
-cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int32_t* ctx_len,
-                          const int64_t* kv_indptr, const int32_t* kv_indices, const uint16_t* k_new,
+// q_indptr (nullable, device int64 [batch+1]): ragged rows, request r has q_indptr[r+1] - q_indptr[r] - 1 drafts <= gamma.
+cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int64_t* q_indptr,
+                          const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices, const uint16_t* k_new,
                           const uint16_t* v_new, const uint8_t* is_migrated, int32_t subset, int32_t* status,
                           cudaStream_t stream);
-cudaError_t launch_commit(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int32_t* ctx_len,
-                          const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
+cudaError_t launch_commit(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int64_t* q_indptr,
+                          const int32_t* ctx_len, const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
                           const int64_t* exp_indptr, const int32_t* exp_indices, int32_t* new_ctx_len, int32_t* status,
                           cudaStream_t stream);
 cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream);
@@ -96,8 +100,8 @@ struct AcceptSplit {
     int32_t rows_cap, vocab_cap, n_sms;
 };
 cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
-                          const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int32_t* ctx_len,
-                          int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
+                          const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int64_t* q_indptr,
+                          const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
                           const AcceptSplit& split, cudaStream_t stream);
 
 cudaError_t launch_accept_logits(const void* logits, int32_t logits_bf16, float temperature, const float* q,

@@ -185,10 +185,11 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     const int head = blockIdx.x - item_idx * Hkv;
     const AttnItem it = a.items[item_idx];
     const int r = it.req;
-    const int gamma = a.gamma;
+    const int gamma = it.gamma;                   // the request's own draft depth
     const int ctx = it.ctx;                       // the plan's copy of ctx_len[r]: one dependent load less before the first tile
     const int n_total = ctx + gamma + 1;          // keys that exist after the append
-    const int M = a.m_rows;
+    const int M = G * (gamma + 1);                // stacked rows of this item (<= the rows the launch is shaped for)
+    const int MS = a.m_stride;                    // rows per partial slot
     const int64_t table0 = it.tbl_off >= 0 ? (int64_t)it.tbl_off : a.kv_indptr[r];
     // a plan checked the table's length on the host; without one (tbl_off < 0) entries past the request's own are not followed
     const int64_t table_end = it.tbl_off >= 0 ? INT64_MAX : a.kv_indptr[r + 1];
@@ -314,7 +315,7 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     for (int j = 0; j < NTW; ++j) {
         const int m = row0 + j * 8 + g;
         const uint16_t* qp = nullptr;
-        if (m < M) qp = a.q + (((int64_t)r * (gamma + 1) + m / G) * Hq + head * G + m % G) * D + tq * 2;
+        if (m < M) qp = a.q + (((int64_t)it.row0 + m / G) * Hq + head * G + m % G) * D + tq * 2;
 #pragma unroll
         for (int kk = 0; kk < KSTEPS; ++kk) {
             qb[kk][j][0] = qp ? __ldg(reinterpret_cast<const uint32_t*>(qp + kk * 16)) : 0u;
@@ -362,7 +363,7 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
                 for (int c = tid; c < n_new * 2 * CPR; c += NT) {
                     const int row = c / (2 * CPR), rem = c - row * (2 * CPR), kv = rem / CPR, ch = rem - kv * CPR;
                     const int p = p_lo + row;
-                    const uint16_t* nsrc = (kv ? a.v_new : a.k_new) + (((int64_t)r * (gamma + 1) + (p - ctx)) * Hkv + head) * D + ch * 8;
+                    const uint16_t* nsrc = (kv ? a.v_new : a.k_new) + (((int64_t)it.row0 + (p - ctx)) * Hkv + head) * D + ch * 8;
                     *reinterpret_cast<int4*>(ks + kv * TILE + (p - key0) * PITCH + ch * 16) = __ldg(reinterpret_cast<const int4*>(nsrc));
                 }
                 __syncthreads();
@@ -546,7 +547,7 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
         }
     __syncthreads();
 
-    const int64_t row_base = (int64_t)r * (gamma + 1);
+    const int64_t row_base = it.row0;
     if (it.part_base < 0) {
         // ---- single chunk: normalise and write bf16, 16 bytes per store
         for (int e = tid; e < M * (D / 8); e += NT) {
@@ -570,8 +571,8 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     // ---- several chunks: store the partial, the last CTA of this (request, head) merges
     {
         const int64_t slot = ((int64_t)it.part_base + it.chunk_idx) * Hkv + head;
-        float* pa = a.part_acc + slot * M * D;
-        float* pm = a.part_ml + slot * M * 2;
+        float* pa = a.part_acc + slot * MS * D;
+        float* pm = a.part_ml + slot * MS * 2;
         for (int e = tid; e < M * (D / 4); e += NT) {
             const int m = e / (D / 4), d4 = e - m * (D / 4);
             *reinterpret_cast<float4*>(pa + (int64_t)m * D + d4 * 4) = *reinterpret_cast<const float4*>(out_s + m * OPITCH + d4 * 4);
@@ -600,7 +601,7 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
 #pragma unroll
         for (int k = 0; k < RB; ++k) mstar[k] = -INFINITY;
         for (int c = 0; c < it.nchunks; ++c) {
-            const float* ml = a.part_ml + (((int64_t)it.part_base + c) * Hkv + head) * M * 2;
+            const float* ml = a.part_ml + (((int64_t)it.part_base + c) * Hkv + head) * MS * 2;
 #pragma unroll
             for (int k = 0; k < RB; ++k) {
                 const int m = mb + k * RP;
@@ -621,8 +622,8 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
                 ml[k] = make_float2(-INFINITY, 0.f);
                 v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (m < M) {
-                    ml[k] = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (slot * M + m) * 2));
-                    v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_acc + (slot * M + m) * D) + d4);
+                    ml[k] = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (slot * MS + m) * 2));
+                    v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_acc + (slot * MS + m) * D) + d4);
                 }
             }
 #pragma unroll
@@ -802,6 +803,8 @@ extern "C" nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_bl
             it.chunk_idx = c;
             it.nchunks = (int32_t)n;
             it.ctx = h_ctx_len[r];
+            it.gamma = gamma;
+            it.row0 = r * (gamma + 1);
             it.tbl_off = -1;                              // this entry point has no host copy of kv_indptr
             items[n_items++] = it;
         }
@@ -840,5 +843,6 @@ extern "C" nsd_status nsd_verify_attn_static(const void* kv_slab, int32_t num_bl
     a.counters = reinterpret_cast<int32_t*>(base + kStaticOffCounters);
     a.status = reinterpret_cast<int32_t*>(base + kStaticOffStatus);
     a.m_rows = rows;
+    a.m_stride = rows;
     return launch_attn(a, st) == cudaSuccess ? NSD_OK : NSD_ERR_CUDA;
 }

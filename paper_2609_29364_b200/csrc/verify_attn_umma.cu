@@ -249,7 +249,8 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
     }
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int Hkv = a.shape.Hkv, Hq = a.shape.Hq, G = Hq / Hkv, gamma = a.gamma, M = a.m_rows;
+    // every unit has its own draft depth: item.gamma + 1 query rows per head, M = G * (item.gamma + 1) stacked rows
+    const int Hkv = a.shape.Hkv, Hq = a.shape.Hq, G = Hq / Hkv, MS = a.m_stride;
     const int64_t n_units = (int64_t)a.n_items * Hkv;
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t wait_limit = a.wait_budget ? a.wait_budget : kSpinLimit;
@@ -323,7 +324,9 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
             if (lane == 0 && k >= 2 && !mbar_wait(smem_u32(&q_empty[qb]), ((k >> 1) - 1) & 1, &abort_s, wait_limit)) okq = false;
             okq = __shfl_sync(0xffffffffu, (int)okq, 0) != 0;
             if (!okq) return false;
-            const int64_t row_base = (int64_t)w.item.req * (gamma + 1);
+            // rows past this unit's M keep whatever an earlier unit left there: finite values on lanes nobody reads
+            const int64_t row_base = w.item.row0;
+            const int M = G * (w.item.gamma + 1);
             const uint32_t qdst = smem0 + kOffQ + qb * kQBytes;
             for (int c = lane; c < M * 16; c += 32) {
                 const int m = c >> 4, ch = c & 15, hh = ch >> 3, cc = ch & 7;
@@ -431,7 +434,7 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
         bool ok = true;
         for (int64_t u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++uidx) {
             const Unit w = load_unit(a, u);
-            const int n_total = w.item.ctx + gamma + 1;
+            const int n_total = w.item.ctx + w.item.gamma + 1;
             // the epilogue has read the previous unit out of the accumulator
             if (lane == 0 && uidx >= 1 && !mbar_wait(smem_u32(&o_empty[(uidx - 1) & 1]), ((uidx - 1) >> 1) & 1, &abort_s, wait_limit)) ok = false;
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -487,7 +490,6 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
         const uint32_t col0 = is_b ? 64u : 0u;              // this warp's score columns, and dims of O in a rescale
         const float sc = rsqrtf(128.f) * kLog2e;
         const int m_row = q * 32 + lane;
-        const bool live = m_row < M;
         uint32_t g = 0, uidx = 0;
         bool fail = false;                                  // warp-uniform: a wait gave up (the CTA is aborting)
         for (int64_t u = blockIdx.x; u < n_units && !fail; u += gridDim.x, ++uidx) {
@@ -495,8 +497,10 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
             const int mr = uidx & 1;                        // which entry of the row statistics this unit uses
             const int ctx = w.item.ctx;                     // the plan's copy: no dependent load at a unit boundary
             const int chunk_end = w.item.blk_end * kBlockSizeU;
-            // keys this row may see: [0, vis_stop); lanes past M hold no row, compute on zeros and are never read
-            const int vis_stop = live ? min(ctx + min(m_row / G, gamma) + 1, chunk_end) : 0x3fffffff;   // lanes past M never mask
+            const int gamma = w.item.gamma;
+            const bool live = m_row < G * (gamma + 1);      // lanes past the unit's rows hold no row and are never read
+            // keys this row may see: [0, vis_stop)
+            const int vis_stop = live ? min(ctx + min(m_row / G, gamma) + 1, chunk_end) : 0x3fffffff;   // lanes without a row never mask
             float m_run = -INFINITY, l_run = 0.f;           // l_run: this warp's half of the keys only
             for (int t = 0; t < w.n_tiles && !fail; ++t, ++g) {
                 const uint32_t sb = g % kSBufs;
@@ -603,13 +607,13 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
         // Thread = one row (TMEM lane te) of O.
         const int te = tid - kWarpEpi0 * 32;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const bool live = te < M;
         uint32_t uidx = 0;
         for (int64_t u = blockIdx.x; u < n_units; u += gridDim.x, ++uidx) {
             const Unit w = load_unit(a, u);
             const int mr = uidx & 1;
-            const int r = w.item.req, head = w.head;
-            const int64_t row_base = (int64_t)r * (gamma + 1);
+            const int head = w.head;
+            const int64_t row_base = w.item.row0;
+            const bool live = te < G * (w.item.gamma + 1);
             const bool mine = mbar_wait(smem_u32(o_full), uidx & 1, &abort_s, wait_limit) &&
                               mbar_wait(smem_u32(&sm_done[mr]), (uidx >> 1) & 1, &abort_s, wait_limit);
             if (epi_bar_or(!mine)) break;                   // a wait gave up: both warps leave together
@@ -635,7 +639,7 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
                 }
                 if (live) {
                     if (split) {
-                        float4* pa = reinterpret_cast<float4*>(a.part_acc + (slot * M + te) * 128 + hh * 64);
+                        float4* pa = reinterpret_cast<float4*>(a.part_acc + (slot * MS + te) * 128 + hh * 64);
 #pragma unroll
                         for (int j = 0; j < 16; ++j)
                             pa[j] = make_float4(__uint_as_float(x[4 * j]), __uint_as_float(x[4 * j + 1]), __uint_as_float(x[4 * j + 2]),
@@ -657,7 +661,7 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
             if (live) {
                 if (split) {
                     // a row that saw no key of this chunk (sum 0, maximum -inf) takes no part in the merge
-                    *reinterpret_cast<float2*>(a.part_ml + (slot * M + te) * 2) = ml;
+                    *reinterpret_cast<float2*>(a.part_ml + (slot * MS + te) * 2) = ml;
                 } else if (a.lse) {
                     a.lse[orow] = (ml.x + log2f(ml.y)) * 0.6931471805599453f;
                 }
@@ -678,24 +682,25 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
 // writes the normalised rows.  Thread = one 4-dim column of one row at a time.
 __global__ void __launch_bounds__(128)
 verify_attn_umma_merge_kernel(const __grid_constant__ AttnLaunch a) {
-    const int Hkv = a.shape.Hkv, Hq = a.shape.Hq, G = Hq / Hkv, M = a.m_rows;
+    const int Hkv = a.shape.Hkv, Hq = a.shape.Hq, G = Hq / Hkv, MS = a.m_stride;
     const int item_idx = blockIdx.x / Hkv, head = blockIdx.x - item_idx * Hkv;
     const AttnItem it = a.items[item_idx];
     if (it.nchunks <= 1 || it.chunk_idx != 0) return;
     const int nch = it.nchunks;
     const int64_t slot0 = (int64_t)it.part_base * Hkv + head;                 // chunk c sits at slot0 + c * Hkv
-    const int64_t row_base = (int64_t)it.req * (a.gamma + 1);
+    const int64_t row_base = it.row0;
+    const int M = G * (it.gamma + 1);
     for (int e = threadIdx.x; e < M * 32; e += 128) {
         const int m = e >> 5, d4 = e & 31;
         float mstar = -INFINITY;
-        for (int c = 0; c < nch; ++c) mstar = fmaxf(mstar, __ldcg(a.part_ml + ((slot0 + (int64_t)c * Hkv) * M + m) * 2));
+        for (int c = 0; c < nch; ++c) mstar = fmaxf(mstar, __ldcg(a.part_ml + ((slot0 + (int64_t)c * Hkv) * MS + m) * 2));
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         float l = 0.f;
 #pragma unroll 4
         for (int c = 0; c < nch; ++c) {
             const int64_t sl = slot0 + (int64_t)c * Hkv;
-            const float2 mlc = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (sl * M + m) * 2));
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_acc + (sl * M + m) * 128) + d4);
+            const float2 mlc = __ldcg(reinterpret_cast<const float2*>(a.part_ml + (sl * MS + m) * 2));
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_acc + (sl * MS + m) * 128) + d4);
             // a row that saw no key of a chunk (sum 0, maximum -inf) takes no part
             const float wgt = mlc.x == -INFINITY ? 0.f : exp2f(mlc.x - mstar);
             acc.x += wgt * v.x;
