@@ -616,8 +616,8 @@ def run_ours(args):
                 "achieved_GBs": (bytes_["round"] - L * bytes_["gather_per_layer"] // 2) / (ms_round_fused * 1e-3) / 1e9,
                 "speedup_over_headline": ms_round / ms_round_fused},
             "mixed_depth_round": {
-                "what": "the same batch with per-request draft depths drawn from [%d, %d] (ragged rows, one attention launch per "
-                        "row-tile class) against the batch padded to depth %d, which is the headline round" % ((cfg.gamma + 1) // 2, cfg.gamma, cfg.gamma),
+                "what": "the same batch with per-request draft depths drawn from [%d, %d] (ragged rows) "
+                        "against the batch padded to depth %d, which is the headline round" % ((cfg.gamma + 1) // 2, cfg.gamma, cfg.gamma),
                 "rows": int(len(rows_idx)), "padded_rows": int(cfg.rows), "ms_per_step": ms_round_ragged,
                 "useful_rows_per_s": n_gpus * len(rows_idx) / (ms_round_ragged * 1e-3),
                 "useful_rows_per_s_padded": n_gpus * len(rows_idx) / (ms_round * 1e-3),

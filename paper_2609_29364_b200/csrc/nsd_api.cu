@@ -14,6 +14,7 @@
 using namespace nsd;
 
 constexpr int kAttnClasses = 6;
+constexpr int kAttnGroups = 2;
 
 struct nsd_ctx {
     nsd_config cfg;
@@ -38,10 +39,12 @@ struct nsd_ctx {
     bool planned;
     int32_t plan_batch, plan_gamma;
     int32_t n_all, n_res, n_mig_items;
-    // Items are grouped by row-tile class (how many 8-row tiles their stacked query rows need: the kernel is instantiated
-    // per class) and, inside a class, ordered longest first.  cls_*[c] .. cls_*[c+1] = the items of class c in the list of
-    // all items, in the resident part and in the reassigned part of the split list.
-    int32_t cls_all[kAttnClasses + 1], cls_res[kAttnClasses + 1], cls_mig[kAttnClasses + 1];
+    // Items whose stacked query rows need at most four 8-row tiles (bound by HBM whatever their width: one launch shaped
+    // for the widest of them) and the wider ones (bound by arithmetic: the tcgen05 engine) form two groups, the wide one
+    // first; inside a group the order is longest first.  grp_*[g] .. grp_*[g+1] = the items of group g in the list of all
+    // items, in the resident part and in the reassigned part of the split list; rows_*[g] = rows of its widest class.
+    int32_t grp_all[kAttnGroups + 1], grp_res[kAttnGroups + 1], grp_mig[kAttnGroups + 1];
+    int32_t rows_all[kAttnGroups], rows_res[kAttnGroups], rows_mig[kAttnGroups];
     int64_t plan_rows;         // query rows of the planned batch: batch * (gamma + 1), or the ragged total
     bool plan_ragged;          // the plan was given per-request depths (h_q_indptr)
     int32_t plan_m_stride;     // rows per split-KV partial slot
@@ -406,7 +409,7 @@ static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, c
     }
     if ((int64_t)items.size() > ctx->max_items || slot > ctx->part_slots) return NSD_ERR_CAPACITY;
     auto longer = [](const Tmp& a, const Tmp& b) {
-        if (a.cls != b.cls) return a.cls > b.cls;                           // the widest row tiles first
+        if ((a.cls >= 4) != (b.cls >= 4)) return a.cls >= 4;                  // the wide group first
         const int la = a.it.blk_end - a.it.blk_begin, lb = b.it.blk_end - b.it.blk_begin;
         if (la != lb) return la > lb;
         if (a.it.req != b.it.req) return a.it.req < b.it.req;
@@ -430,21 +433,24 @@ static nsd_status verify_plan_impl(nsd_ctx* ctx, int32_t batch, int32_t gamma, c
     }
     NSD_CUDA(ctx, cudaEventRecord(ctx->ev_plan_free, st));
     {
-        // class boundaries of the three lists (classes run from the widest to the narrowest)
-        auto bounds = [&](int32_t* off, int mig_filter) {
-            int32_t count[kAttnClasses] = {0};
+        // group boundaries of the three lists and the widest class of each group
+        auto bounds = [&](int32_t* off, int32_t* rows, int mig_filter) {
+            int32_t count[kAttnGroups] = {0, 0};
+            int widest[kAttnGroups] = {-1, -1};
             for (const Tmp& t : items)
-                if (mig_filter < 0 || t.mig == mig_filter) count[t.cls]++;
-            int32_t run = 0;
-            for (int c = kAttnClasses - 1; c >= 0; --c) {                 // position c' = kAttnClasses - 1 - c in list order
-                off[kAttnClasses - 1 - c] = run;
-                run += count[c];
-            }
-            off[kAttnClasses] = run;
+                if (mig_filter < 0 || t.mig == mig_filter) {
+                    const int g = t.cls >= 4 ? 0 : 1;                       // list position: wide group first
+                    count[g]++;
+                    widest[g] = std::max(widest[g], t.cls);
+                }
+            off[0] = 0;
+            off[1] = count[0];
+            off[2] = count[0] + count[1];
+            for (int g = 0; g < kAttnGroups; ++g) rows[g] = widest[g] >= 0 ? attn_class_rows(widest[g]) : 0;
         };
-        bounds(ctx->cls_all, -1);
-        bounds(ctx->cls_res, 0);
-        bounds(ctx->cls_mig, 1);
+        bounds(ctx->grp_all, ctx->rows_all, -1);
+        bounds(ctx->grp_res, ctx->rows_res, 0);
+        bounds(ctx->grp_mig, ctx->rows_mig, 1);
     }
     ctx->plan_rows = row0[batch];
     ctx->plan_ragged = h_q_indptr != nullptr;
@@ -554,8 +560,9 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
     a.wait_budget = ctx->wait_budget;
     a.any_split = ctx->plan_split_slots > 0;
     const AttnItem* base = subset == 0 ? ctx->d_items_all : (subset == 1 ? ctx->d_items_split : ctx->d_items_split + ctx->n_res);
-    const int32_t* cls = subset == 0 ? ctx->cls_all : (subset == 1 ? ctx->cls_res : ctx->cls_mig);
-    if (cls[kAttnClasses] == 0) return NSD_OK;
+    const int32_t* grp = subset == 0 ? ctx->grp_all : (subset == 1 ? ctx->grp_res : ctx->grp_mig);
+    const int32_t* grp_rows = subset == 0 ? ctx->rows_all : (subset == 1 ? ctx->rows_res : ctx->rows_mig);
+    if (grp[kAttnGroups] == 0) return NSD_OK;
     if ((ctx->attn_feed_tma || ctx->attn_tcgen05) && !fuse && ctx->cfg.head_dim == 128) {
         const int slab = layer % ctx->cfg.num_slabs;
         if (ctx->tmap_slab[slab] != a.pool_slab) {
@@ -572,13 +579,13 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
         }
         a.tma_feed = ctx->attn_feed_tma;
     }
-    // one launch per row-tile class present (a batch of one draft depth has one), widest first
-    for (int pos = 0; pos < kAttnClasses; ++pos) {
-        const int n = cls[pos + 1] - cls[pos];
+    // one launch per group present (a batch of one draft depth has one), each shaped for its widest item
+    for (int pos = 0; pos < kAttnGroups; ++pos) {
+        const int n = grp[pos + 1] - grp[pos];
         if (n == 0) continue;
-        a.items = base + cls[pos];
+        a.items = base + grp[pos];
         a.n_items = n;
-        a.m_rows = std::min(attn_class_rows(kAttnClasses - 1 - pos), ctx->plan_m_stride);
+        a.m_rows = std::min(grp_rows[pos], ctx->plan_m_stride);
         if (a.tmap_valid && ctx->attn_tcgen05 && attn_umma_supported(a) && (ctx->attn_tcgen05 == 2 || attn_umma_preferred(a))) {
             NSD_CUDA(ctx, launch_attn_umma(a, st, ctx->n_sms));
             ctx->launches += a.any_split ? 2 : 1;                            // the engine's merge kernel follows when a request is split

@@ -1,5 +1,5 @@
 """GPU parity of per-request draft depths (ragged rows): one batch mixes depths 0..gamma, nothing is padded.  The whole
-round (gather, append, attention in one launch per row-tile class, acceptance), its gather-through variant, the
+round (gather, append, attention in one launch per group of row widths, acceptance), its gather-through variant, the
 host-buffer variant and the suffix commit against the oracle: pool bit for bit, attention within tolerance, accepted
 lengths and tokens exact."""
 import numpy as np
@@ -130,7 +130,7 @@ def _run(cfg, slabs, fuse=False, host_variant=False, chunk_blocks=0, split_flag=
 
 @pytest.mark.parametrize("split_flag", [1 << 4, 1 << 5], ids=["split_first", "wait_first"])
 def test_mixed_depths_round(split_flag):
-    """Depths 0..8 at the Qwen3-8B group size: 4..36 stacked rows, i.e. five row-tile classes, the widest on the tcgen05 engine."""
+    """Depths 0..8 at the Qwen3-8B group size: 4..36 stacked rows, the widest on the tcgen05 engine, the rest in one mma.sync launch."""
     _run(MIX, 2, split_flag=split_flag)
 
 
