@@ -118,7 +118,7 @@ Layout make_layout(const nsd_config* c) {
     L.status = off;      off = align_up(off + 4 * sizeof(int32_t), 256);
     L.counters = off;    off = align_up(off + (size_t)c->max_batch * c->num_kv_heads * sizeof(int32_t), 256);
     L.acc_rows = std::min<int32_t>(c->max_batch, 512);                   // requests that may be shared among acceptance CTAs
-    L.acc_counters = off; off = align_up(off + (size_t)L.acc_rows * sizeof(int32_t), 256);
+    L.acc_counters = off; off = align_up(off + (size_t)(L.acc_rows + 2) * sizeof(int32_t), 256);   // + the two request tickets of the logits kernel
     L.items_all = off;   off = align_up(off + (size_t)L.max_items * sizeof(AttnItem), 256);
     L.items_split = off; off = align_up(off + (size_t)L.max_items * sizeof(AttnItem), 256);
     L.acc_scratch = off; off = align_up(off + (size_t)L.acc_rows * ((c->vocab_size + 127) / 128) * sizeof(double), 256);
@@ -642,7 +642,8 @@ nsd_status nsd_spec_accept_logits(nsd_ctx* ctx, const void* logits, int32_t logi
     if ((new_ctx_len != nullptr) && !ctx_len) return NSD_ERR_INVALID_ARG;
     NSD_CUDA(ctx, launch_accept_logits(logits, logits_dtype, temperature, q, draft_tok, u_acc, u_smp, batch, gamma, vocab,
                                        gamma_r, ctx_len, acc_len, out_tok, new_ctx_len, ctx->d_status, ctx->n_sms,
-                                       ctx->logits_feed, static_cast<cudaStream_t>(stream)));
+                                       ctx->logits_feed, ctx->accept_split.counters + ctx->accept_split.rows_cap,
+                                       static_cast<cudaStream_t>(stream)));
     ctx->launches++;
     return NSD_OK;
 }

@@ -109,6 +109,6 @@ cudaError_t launch_accept_logits(const void* logits, int32_t logits_bf16, float 
                                  int32_t gamma, int32_t vocab, const int32_t* gamma_r, const int32_t* ctx_len,
                                  int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
                                  int32_t n_sms, int32_t feed /* 0 = direct loads, 1 = shared-memory ring where aligned */,
-                                 cudaStream_t stream);
+                                 int32_t* tickets /* two words, zero between launches */, cudaStream_t stream);
 
 }  // namespace nsd

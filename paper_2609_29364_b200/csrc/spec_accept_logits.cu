@@ -3,7 +3,10 @@
 // while u < min(1, p/q), residual resampling, bonus token) is fused into the kernel, so
 // the [batch][gamma+1][vocab] probability tensor is never written or re-read.
 //
-// One CTA per request.  Rows are swept in order and only as far as needed: row i costs
+// One CTA at a time per request; a persistent grid of one CTA (1024 threads) per SM takes the requests from a
+// counter.  That bounds the rows in flight to one per SM (~90 MB at the Qwen3 vocabulary), so the draw's second
+// read of the rejected row finds it in L2; with a CTA per request and four resident per SM, 512 rows (~310 MB) were
+// in flight and that read went to DRAM again.  Rows are swept in order and only as far as needed: row i costs
 // one pass (block-wide max and sum of exponentials, kept online per thread and merged
 // through shared memory), after which warp 0 can test draft i; the first rejection ends
 // the sweep.  The draw then re-reads row n (an L2 hit: one row is ~0.6 MB) together with
@@ -16,18 +19,20 @@
 //
 // Feed.  Where rows start on 16-byte boundaries and hold whole 16-byte pieces (vocab a multiple of
 // 4 for fp32, of 8 for bf16) they do not travel through registers one load at a time: every
-// thread copies its own 16-byte pieces of the next tiles with cp.async into a ring of 8 KiB tiles in shared memory and reads them back
-// itself, so a CTA keeps 32-96 KiB in flight with no barrier of any kind and no registers
+// thread copies its own 16-byte pieces of the next tiles with cp.async into a ring of 16 KiB tiles in shared memory and reads them back
+// itself, so a CTA keeps up to 176 KiB in flight with no barrier of any kind and no registers
 // held.  Each thread sees the same elements in the same order as with direct loads, so the two
 // feeds give identical results; other shapes use direct loads.
 #include <cuda_bf16.h>
+
+#include <algorithm>
 
 #include "nsd_internal.h"
 
 namespace nsd {
 namespace {
 
-constexpr int kThreads = 512;
+constexpr int kThreads = 1024;                  // one CTA per SM (see the kernel): all of an SM's loads come from it
 constexpr int kWarps = kThreads / 32;
 constexpr int kSeg = 128;                       // tokens per segment of the draw
 constexpr int kAhead = 32;                      // drafts per request whose scalars are fetched ahead
