@@ -563,7 +563,7 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
     const int32_t* grp = subset == 0 ? ctx->grp_all : (subset == 1 ? ctx->grp_res : ctx->grp_mig);
     const int32_t* grp_rows = subset == 0 ? ctx->rows_all : (subset == 1 ? ctx->rows_res : ctx->rows_mig);
     if (grp[kAttnGroups] == 0) return NSD_OK;
-    if ((ctx->attn_feed_tma || ctx->attn_tcgen05) && !fuse && ctx->cfg.head_dim == 128) {
+    if ((ctx->attn_feed_tma || ctx->attn_tcgen05) && ctx->cfg.head_dim == 128) {
         const int slab = layer % ctx->cfg.num_slabs;
         if (ctx->tmap_slab[slab] != a.pool_slab) {
             ctx->tmap_slab[slab] = make_kv_tensor_map(&ctx->tmaps[slab], a.pool_slab, ctx->shape) ? a.pool_slab : nullptr;

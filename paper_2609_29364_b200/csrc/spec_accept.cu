@@ -192,7 +192,7 @@ __device__ __forceinline__ void spec_accept_body(const AcceptArgs& a) {
         __syncthreads();
     };
 
-    if (SPLIT) {
+    if constexpr (SPLIT) {
         // this CTA's slice goes to the scratch row; whoever arrives last owns the rest of the work
         double* row = a.seg_scratch + (int64_t)r * n_seg;
         const int per = (n_seg + a.split - 1) / a.split;
@@ -209,17 +209,50 @@ __device__ __forceinline__ void spec_accept_body(const AcceptArgs& a) {
         if (!s_last) return;
         __threadfence();
         for (int s = tid; s < n_seg; s += kAcceptThreads) seg_sum[s] = __ldcg(row + s);
-    } else {
-        sweep(0, n_seg, nullptr, residual);
-    }
-    __syncthreads();
-    prefix();
-    if (residual && s_total == 0.0) {           // empty residual: draw from the target row instead
-        residual = false;
-        __syncthreads();
-        sweep(0, n_seg, nullptr, false);
         __syncthreads();
         prefix();
+        if (residual && s_total == 0.0) {       // empty residual: draw from the target row instead
+            residual = false;
+            __syncthreads();
+            sweep(0, n_seg, nullptr, false);
+            __syncthreads();
+            prefix();
+        }
+    } else {
+        // one CTA owns the request: the sweep written out in place with `residual` a run-time flag (the templated
+        // sweep costs this instantiation the 32 registers that let four CTAs share an SM)
+        constexpr int n_warps = kAcceptThreads / 32;
+        for (int attempt = 0; attempt < 2; ++attempt) {
+            for (int s = warp; s < n_seg; s += n_warps) {
+                const int k0 = s * kSeg + lane * 4;
+                double acc = 0.0;
+                if (vec_ok) {
+                    if (k0 < vocab) {
+                        const float4 pv = __ldg(reinterpret_cast<const float4*>(prow + k0));
+                        float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (residual) qv = __ldg(reinterpret_cast<const float4*>(qrow + k0));
+                        acc = (double)weight(pv.x, qv.x, residual);
+                        acc += (double)weight(pv.y, qv.y, residual);
+                        acc += (double)weight(pv.z, qv.z, residual);
+                        acc += (double)weight(pv.w, qv.w, residual);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (k0 + j < vocab) acc += (double)weight(prow[k0 + j], residual ? qrow[k0 + j] : 0.f, residual);
+                }
+                acc = warp_sum(acc);
+                if (lane == 0) seg_sum[s] = acc;
+            }
+            __syncthreads();
+            prefix();
+            if (residual && s_total == 0.0) {   // empty residual: draw from the target row instead
+                residual = false;
+                __syncthreads();
+                continue;
+            }
+            break;
+        }
     }
 
     const double total = s_total;
@@ -275,7 +308,8 @@ __device__ __forceinline__ void spec_accept_body(const AcceptArgs& a) {
         int32_t v = -1;
         if (tid < n) v = tok_req[tid];
         else if (tid == n) v = s_token;
-        a.out_tok[row0 + tid] = v;
+        // (the row offset is read again rather than kept in registers across the sweep)
+        a.out_tok[(a.q_indptr ? a.q_indptr[r] : (int64_t)r * (a.gamma + 1)) + tid] = v;
     }
     if (tid == 0) {
         a.acc_len[r] = n;

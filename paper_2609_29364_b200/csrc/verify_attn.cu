@@ -128,6 +128,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
                  : "memory");
 }
+// One box back to global memory (a bulk group of the issuing thread); x, y as for the load, never negative.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int32_t x, int32_t y, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+}
 
 // Shared-memory tiles are [rows][D] bf16 with every row padded by 16 bytes: eight
 // consecutive rows then start 16 bytes apart modulo 128, so the eight row reads of
@@ -153,7 +157,9 @@ struct Smem {
 
 // NW warps, each serving NTW tiles of 8 query rows; rows m >= M are zero padding.  TMA = the K/V tiles arrive by
 // cp.async.bulk.tensor boxes (one warp, head_dim 128, one pool block per stage, no gather-through) instead of cp.async.
-template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false>
+// FUSE (TMA-fed variant only; the cp.async variant decides at run time): compiled with the gather-through path.  A
+// separate instantiation, because carrying the path unused cost the plain kernel 5 % (registers, instruction fetch).
+template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false, bool FUSE = false>
 __global__ void __launch_bounds__(NW * 32)
 verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     static_assert(!TMA || (D == 128 && TK == 16), "the TMA-fed variant covers head_dim 128 with one pool block per stage");
@@ -198,7 +204,7 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
 
     // Gather-through: a reassigned request streams its committed KV from the source blocks and writes it,
     // with the new tokens, to its destination blocks on the way (uniform per CTA).
-    const bool fused = !TMA && a.fuse != 0 && it.src_off >= 0;
+    const bool fused = (TMA ? FUSE : a.fuse != 0) && it.src_off >= 0;
     const int n_src = (ctx + kBlockSize - 1) / kBlockSize;       // blocks that hold committed KV
     int32_t* dst_s = blk_s + SM::kMaxChunkBlocks;
 
@@ -261,11 +267,21 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
             // four boxes of 16 keys x 64 dims (K lo, K hi, V lo, V hi), one per lane, completing on the stage's barrier
             if (t < n_tiles && warp == 0) {
                 const uint32_t bar = smem_u32(&full_bar[stage]);
-                if (lane == 0) mbar_expect_tx(bar, STAGE);
-                __syncwarp();
-                if (lane < 4) {
-                    const int32_t row = ((blk_s[t] * 2 + (lane >> 1)) * Hkv + head) * kBlockSize;
-                    tma_load_2d(smem0 + stage * STAGE + lane * 2048, &a.tmap, (lane & 1) * 64, row, bar);
+                // gather-through: the stage's previous tile may still be on its way out to its destination block
+                if (fused && lane < 4) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                if (blk_s[t] >= 0) {
+                    if (lane == 0) mbar_expect_tx(bar, STAGE);
+                    __syncwarp();
+                    if (lane < 4) {
+                        const int32_t row = ((blk_s[t] * 2 + (lane >> 1)) * Hkv + head) * kBlockSize;
+                        tma_load_2d(smem0 + stage * STAGE + lane * 2048, &a.tmap, (lane & 1) * 64, row, bar);
+                    }
+                } else {
+                    // a fresh block (gather-through only): nothing to read.  V must be finite (zero); K is masked or injected.
+                    __syncwarp();
+                    for (int c = lane; c < 256; c += 32) *reinterpret_cast<int4*>(smem + stage * STAGE + 4096 + c * 16) = make_int4(0, 0, 0, 0);
+                    __syncwarp();
+                    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
                 }
             }
             return;
@@ -354,7 +370,50 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
         issue_tile(t + kStages - 1, (stage + kStages - 1) % kStages);
         const int key0 = key0_chunk + t * TK;
         const bool need_mask = key0 + TK > ctx + 1;   // some key of the tile is hidden from some row
-        if (fused) {
+        if constexpr (TMA) {
+            if (fused) {
+                // Tiles sit as [K lo | K hi | V lo | V hi], each [16 keys][64 dims] with the 128-byte swizzle: the 16-byte
+                // chunk c of row r of a part is at r * 128 + ((c ^ (r & 7)) << 4).
+                unsigned char* ts = smem + stage * STAGE;
+                const int p_lo = max(ctx, key0), p_hi = min(ctx + gamma, key0 + TK - 1);
+                if (p_lo <= p_hi) {
+                    // new tokens of this request that fall into the tile come from k_new / v_new, not from the pool
+                    const int n_new = p_hi - p_lo + 1;
+                    for (int c = tid; c < n_new * 32; c += NT) {
+                        const int row = c >> 5, rem = c & 31, kv = rem >> 4, ch = rem & 15;
+                        const int p = p_lo + row, rr = p - key0;
+                        const uint16_t* nsrc = (kv ? a.v_new : a.k_new) + (((int64_t)it.row0 + (p - ctx)) * Hkv + head) * D + ch * 8;
+                        *reinterpret_cast<int4*>(ts + (kv * 2 + (ch >> 3)) * 2048 + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) =
+                            __ldg(reinterpret_cast<const int4*>(nsrc));
+                    }
+                    __syncthreads();
+                }
+                if (blk_s[t] >= 0) {
+                    // the whole tile goes to its destination block: four boxes, straight out of the stage
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncthreads();
+                    if (warp == 0 && lane < 4) {
+                        const int32_t row = ((dst_s[t] * 2 + (lane >> 1)) * Hkv + head) * kBlockSize;
+                        tma_store_2d(&a.tmap, (lane & 1) * 64, row, smem0 + stage * STAGE + lane * 2048);
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        // slots past the last token are about to be zeroed for the arithmetic: the copy must have read them
+                        // first, because the destination block gets the source's tail slots verbatim
+                        if (key0 + TK > n_total) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    }
+                    if (key0 + TK > n_total) __syncthreads();
+                } else if (p_lo <= p_hi) {
+                    // a fresh block: only the new tokens' rows are written, the other slots keep what they held
+                    const int n_new = p_hi - p_lo + 1;
+                    uint16_t* dbase = a.pool_slab_w + (int64_t)dst_s[t] * block_elems + (int64_t)head * (kBlockSize * D);
+                    for (int c = tid; c < n_new * 32; c += NT) {
+                        const int row = c >> 5, rem = c & 31, kv = rem >> 4, ch = rem & 15;
+                        const int rr = p_lo + row - key0;
+                        const int4 v = *reinterpret_cast<const int4*>(ts + (kv * 2 + (ch >> 3)) * 2048 + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4));
+                        *reinterpret_cast<int4*>(dbase + (int64_t)kv * v_off + rr * D + ch * 8) = v;
+                    }
+                }
+            }
+        } else if (fused) {
             unsigned char* ks = smem + stage * STAGE;
             // new tokens of this request that fall into the tile come from k_new / v_new, not from the pool
             const int p_lo = max(ctx, key0), p_hi = min(ctx + gamma, key0 + TK - 1);
@@ -514,6 +573,10 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
         return;
     }
     cp_async_wait<0>();
+    if constexpr (TMA) {
+        // gather-through: the last tiles may still be on their way out of the ring
+        if (fused && warp == 0 && lane < 4) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    }
     __syncthreads();                                      // the ring is free: reuse it to stage the output
 
     // ---- row sums across the 8 lanes that share tq
@@ -653,16 +716,16 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     }
 }
 
-template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false>
+template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false, bool FUSE = false>
 cudaError_t launch_one(const AttnLaunch& a, cudaStream_t stream) {
     const int64_t grid = (int64_t)a.n_items * a.shape.Hkv;
-    verify_attn_kernel<D, NW, NTW, TK, kStages, TMA><<<(unsigned)grid, NW * 32, Smem<D, TK, kStages, NW * NTW * 8, TMA>::kBytes, stream>>>(a);
+    verify_attn_kernel<D, NW, NTW, TK, kStages, TMA, FUSE><<<(unsigned)grid, NW * 32, Smem<D, TK, kStages, NW * NTW * 8, TMA>::kBytes, stream>>>(a);
     return cudaGetLastError();
 }
 
-template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false>
+template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false, bool FUSE = false>
 cudaError_t init_one() {
-    return cudaFuncSetAttribute(verify_attn_kernel<D, NW, NTW, TK, kStages, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(verify_attn_kernel<D, NW, NTW, TK, kStages, TMA, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 Smem<D, TK, kStages, NW * NTW * 8, TMA>::kBytes);
 }
 
@@ -682,7 +745,8 @@ cudaError_t attn_init() {
     NSD_ATTN_SHAPES(NSD_INIT, 64, kStagesD64)
     NSD_ATTN_SHAPES(NSD_INIT, 128, kStagesD128)
 #define NSD_INIT_TMA(DD, WW, TT, KK, SS) \
-    if ((e = init_one<DD, WW, TT, KK, SS, true>()) != cudaSuccess) return e;
+    if ((e = init_one<DD, WW, TT, KK, SS, true>()) != cudaSuccess) return e; \
+    if ((e = init_one<DD, WW, TT, KK, SS, true, true>()) != cudaSuccess) return e;
     NSD_ATTN_SHAPES(NSD_INIT_TMA, 128, kStagesD128)
 #undef NSD_INIT_TMA
 #undef NSD_INIT
@@ -697,9 +761,9 @@ cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
     // K/V tiles by tensor copies where that measured faster: the shapes that are bound by HBM (up to 32 stacked rows:
     // +4-6 % at 20-24 rows, +3 % at 28-32).  The five- and six-row-tile shapes are bound by the tensor pipe and by
     // shared-memory reads and ran 8-25 % slower fed this way, so they stay on cp.async.
-    if (a.tma_feed && a.tmap_valid && !a.fuse && a.shape.D == 128 && (nw == 1 || (nw == 2 && ntw == 2))) {
+    if (a.tma_feed && a.tmap_valid && a.shape.D == 128 && (nw == 1 || (nw == 2 && ntw == 2))) {
 #define NSD_TMA_CASE(DD, WW, TT, KK, SS) \
-        if (nw == WW && ntw == TT) return launch_one<DD, WW, TT, KK, SS, true>(a, stream);
+        if (nw == WW && ntw == TT) return a.fuse ? launch_one<DD, WW, TT, KK, SS, true, true>(a, stream) : launch_one<DD, WW, TT, KK, SS, true>(a, stream);
         NSD_ATTN_SHAPES(NSD_TMA_CASE, 128, kStagesD128)
 #undef NSD_TMA_CASE
     }
