@@ -365,10 +365,15 @@ nsd_status nsd_verify_round(nsd_ctx* ctx, const nsd_round_args* args, void* stre
  * (pinned for full speed): every input of `h` except kv_pool is copied to the
  * matching buffer of `d` on `stream`, the round runs, and o, acc_len, out_tok
  * (and new_ctx_len when both are non-null) are copied back into `h`'s buffers;
- * the call synchronises `stream` before returning.  The acceptance inputs (p,
- * q_draft, draft_tok, u_acc, u_smp) travel on an internal copy stream while the
- * layers run, and o is read back before the acceptance is enqueued, so the
- * transfers overlap the kernels.  `h->kv_pool` is ignored:
+ * the call synchronises `stream` before returning.  The acceptance inputs
+ * (draft_tok, u_acc, u_smp) travel on an internal copy stream while the layers
+ * run, and o is read back before the acceptance is enqueued, so the transfers
+ * overlap the kernels.  p and q_draft, by far the largest inputs, are copied the
+ * same way unless `h`'s buffers are pinned host memory the device can address
+ * (cudaHostAlloc / cudaHostRegister): then they stay where they are and the
+ * acceptance kernel reads the gamma scalars and the one row (pair) per request
+ * it needs over the link (d->p, d->q_draft may then be null); the bytes it read
+ * are counted in *h2d_bytes.  `h->kv_pool` is ignored:
  * the pool is worker state that stays on the device.  h_* table arguments of
  * the plan are taken from `h` (ctx_len, kv_indptr, is_migrated), so no separate
  * nsd_verify_plan call is needed.  Bytes moved are written to the two counters

@@ -809,9 +809,23 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
         {h->mig_dst, d->mig_dst, h->n_mig_blocks * 4},
         {h->q_indptr, d->q_indptr, h->q_indptr ? (batch + 1) * 8LL : 0},
     };
+    // The probability tensors are by far the largest inputs (2.8 GB at batch 512 and the Qwen3 vocabulary), yet the
+    // acceptance reads gamma scalars and one row (pair) per request of them.  Where the caller's buffers are pinned host
+    // memory that the device can address, they are not copied: the acceptance kernel reads what it needs over the link.
+    auto device_view = [](const void* hp) -> const void* {
+        cudaPointerAttributes at{};
+        if (!hp || cudaPointerGetAttributes(&at, hp) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+    };
+    const float* p_direct = static_cast<const float*>(device_view(h->p));
+    const float* q_direct = static_cast<const float*>(device_view(h->q_draft));
+    const bool direct = p_direct && q_direct;
     const Copy accept_in[] = {
-        {h->p, d->p, rows * V * 4},
-        {h->q_draft, d->q_draft, drafts * V * 4},
+        {h->p, d->p, direct ? 0 : rows * V * 4},
+        {h->q_draft, d->q_draft, direct ? 0 : drafts * V * 4},
         {h->draft_tok, d->draft_tok, drafts * 4},
         {h->u_acc, d->u_acc, drafts * 4},
         {h->u_smp, d->u_smp, batch * 4LL},
@@ -820,6 +834,7 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
         if (c.bytes != 0 && (!c.src || !c.dst)) return NSD_ERR_INVALID_ARG;
     for (const Copy& c : accept_in)
         if (c.bytes != 0 && (!c.src || !c.dst)) return NSD_ERR_INVALID_ARG;
+    if (!h->p || !h->q_draft || (!direct && (!d->p || !d->q_draft))) return NSD_ERR_INVALID_ARG;
     if (!h->k_new || !d->k_new || !h->v_new || !d->v_new || !h->q || !d->q) return NSD_ERR_INVALID_ARG;
     if (!h->o || !d->o || !h->acc_len || !d->acc_len || !h->out_tok || !d->out_tok) return NSD_ERR_INVALID_ARG;
     nsd_status s = nsd_verify_plan(ctx, batch, gamma, h->ctx_len, h->kv_indptr, h->is_migrated, h->q_indptr, 0, stream);
@@ -844,7 +859,12 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
     for (const Copy& c : accept_in) NSD_CUDA(ctx, upload(c));
     NSD_CUDA(ctx, cudaEventRecord(ctx->ev_accept_in, ctx->copy));
     const BeforeAccept hook{h->o, (size_t)q_layer_bytes, ctx->ev_accept_in};
-    s = round_impl(ctx, d, stream, &hook);
+    nsd_round_args dd = *d;
+    if (direct) {
+        dd.p = p_direct;
+        dd.q_draft = q_direct;
+    }
+    s = round_impl(ctx, &dd, stream, &hook);
     if (s != NSD_OK) {
         cudaStreamSynchronize(ctx->copy);
         cudaStreamSynchronize(ctx->down);
@@ -862,6 +882,14 @@ nsd_status nsd_verify_round_host(nsd_ctx* ctx, const nsd_round_args* h, const ns
         down += c.bytes;
     }
     NSD_CUDA(ctx, cudaStreamSynchronize(st));
+    if (direct) {
+        // what the acceptance kernel read over the link: per request the gathers of its tests and the one row (pair) of the draw
+        for (int r = 0; r < batch; ++r) {
+            const int64_t g_r = h->q_indptr ? h->q_indptr[r + 1] - h->q_indptr[r] - 1 : gamma;
+            const int64_t n = h->acc_len[r];
+            up += (n < g_r ? 2 : 1) * V * 4 + 2 * 4 * std::min<int64_t>(g_r, n + 1);
+        }
+    }
     if (h2d_bytes) *h2d_bytes = up;
     if (d2h_bytes) *d2h_bytes = down;
     return NSD_OK;

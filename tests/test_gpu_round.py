@@ -27,7 +27,7 @@ def _oracle_round(cfg, meta, pool0, k_new, v_new, q, acc_in):
     return pool, outs, acc, out, new_ctx
 
 
-def _run_round(cfg, slabs, host_variant=False, repeat=1, fuse=False, plan_without_flags=False):
+def _run_round(cfg, slabs, host_variant=False, repeat=1, fuse=False, plan_without_flags=False, pageable_probs=False):
     """The first-layer order is a flag of the context: the tests below set it to cover both orders."""
     meta = W.make_batch_meta(cfg)
     pool0 = np.stack([W.pool_layer(cfg, meta, s) for s in range(slabs)])
@@ -50,11 +50,13 @@ def _run_round(cfg, slabs, host_variant=False, repeat=1, fuse=False, plan_withou
     stream = torch.cuda.Stream()
     if host_variant:
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a.view(np.int16) if a.dtype == np.uint16 else a)).pin_memory()
+        # pinned probability tensors are read in place by the acceptance kernel; pageable ones are copied like the rest
+        probs = (lambda a: torch.from_numpy(np.ascontiguousarray(a))) if pageable_probs else pin
         h = dict(kv_pool=None, n_mig_blocks=db.n_mig_blocks, mig_src=pin(meta.mig_src) if db.n_mig_blocks else None,
                  mig_dst=pin(meta.mig_dst) if db.n_mig_blocks else None, batch=B, gamma=cfg.gamma,
                  ctx_len=pin(meta.ctx_len), kv_indptr=pin(meta.kv_indptr), kv_indices=pin(meta.kv_indices),
                  is_migrated=pin(meta.is_migrated), k_new=pin(k_new), v_new=pin(v_new), q=pin(q),
-                 o=torch.zeros(q.shape, dtype=torch.int16).pin_memory(), p=pin(p), q_draft=pin(qd), draft_tok=pin(tok),
+                 o=torch.zeros(q.shape, dtype=torch.int16).pin_memory(), p=probs(p), q_draft=probs(qd), draft_tok=pin(tok),
                  u_acc=pin(ua), u_smp=pin(us), acc_len=torch.zeros(B, dtype=torch.int32).pin_memory(),
                  out_tok=torch.zeros((B, g1), dtype=torch.int32).pin_memory(),
                  new_ctx_len=torch.zeros(B, dtype=torch.int32).pin_memory(), fuse_gather=int(fuse))
@@ -68,7 +70,9 @@ def _run_round(cfg, slabs, host_variant=False, repeat=1, fuse=False, plan_withou
             for _ in range(repeat):
                 up, down = ctx.nsd_verify_round_host(ctx.round_args(**h), ctx.round_args(**d), int(meta.kv_indptr[-1]),
                                                      stream=stream)
-        assert up > p.nbytes and down >= q.nbytes
+        layers_in = k_new.nbytes + v_new.nbytes + q.nbytes
+        assert up > layers_in and down >= q.nbytes
+        assert (up > layers_in + p.nbytes + qd.nbytes) == pageable_probs      # copied whole, or read in place row by row
         o_gpu, acc_g, out_g, new_g = h["o"].numpy().view(np.uint16), h["acc_len"].numpy(), h["out_tok"].numpy(), h["new_ctx_len"].numpy()
     else:
         with torch.cuda.stream(stream):
@@ -125,6 +129,7 @@ def test_round_twice_gives_the_same_state(split, monkeypatch):
 def test_host_buffer_round(split, monkeypatch):
     monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", SPLIT_FLAG[split])
     _run_round(MULTI, 2, host_variant=True)
+    _run_round(MULTI, 2, host_variant=True, pageable_probs=True)
     _run_round(W.CONFIGS["tiny"], 1, host_variant=True, repeat=2)
 
 
