@@ -37,6 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 # profiler capture of a smaller case of the same kernel (709.4 MB over 698.9 MB for one whole-batch pass); the
 # full-size launch is too large to capture under the profiler, and traffic grows with the keys streamed.
 ATTN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.015
+# The same for verify_attn_umma_kernel, the engine the library picks from 33 stacked query rows per kv head on
+# (2058 MB over 2036 MB for one whole-batch pass of a small long-context case; its merge kernel is timed with it).
+UMMA_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.011
 
 
 def parse_args():
@@ -448,6 +451,13 @@ def run_ours(args):
     ms_attn_launch = timed(attn_all_layers, args.steps, args.warmup) / L
     peak, peak_kind = measured_peak()
     attn_gbs = bytes_["attn_per_layer"] / (ms_attn_launch * 1e-3) / 1e9
+    # which engine the library launches for this batch: the tcgen05 one from 33 stacked query rows per kv head on
+    # (unless the context's flags say otherwise), else the mma.sync one
+    stacked_rows = (cfg.num_q_heads // cfg.num_kv_heads) * (cfg.gamma + 1)
+    use_umma = bool(cfg.head_dim == 128 and cfg.block_size == 16 and stacked_rows <= 64 and
+                    ((stacked_rows > 32 and not (args.ctx_flags & 4)) or (args.ctx_flags & 2)))
+    attn_kernel_name = "verify_attn_umma_kernel + its merge kernel" if use_umma else "verify_attn_kernel"
+    attn_traffic_ratio = UMMA_TRAFFIC_PER_ALGORITHMIC_BYTE if use_umma else ATTN_TRAFFIC_PER_ALGORITHMIC_BYTE
 
     # ---- the other kernels alone and the round without any reassigned request (exposed prepare time)
     def prepare_all_layers():
@@ -589,10 +599,10 @@ def run_ours(args):
             "committed_tokens_per_s": n_gpus * committed / (ms_round * 1e-3),
             "verified_rows_per_s": n_gpus * cfg.rows / (ms_round * 1e-3),
             "mean_accepted_len": float(acc_len.mean()),
-            "roofline": {"kernel": "verify_attn_kernel (one launch per layer, timed alone)", "bound": "hbm",
+            "roofline": {"kernel": attn_kernel_name + " (one launch per layer, timed alone)", "bound": "hbm",
                          "achieved": attn_gbs, "peak": peak, "peak_kind": f"{peak_kind} copy bandwidth",
                          "unit": "GB/s", "frac": attn_gbs / peak, "frac_of_nominal_8TBs": attn_gbs / NOMINAL_HBM_GBS,
-                         "traffic": int(ATTN_TRAFFIC_PER_ALGORITHMIC_BYTE * bytes_["attn_per_layer"]),
+                         "traffic": int(attn_traffic_ratio * bytes_["attn_per_layer"]),
                          "traffic_source": "profiler capture of a smaller case of the same kernel, scaled by algorithmic bytes",
                          "bytes_per_launch": bytes_["attn_per_layer"], "ms_per_launch": ms_attn_launch},
             "round_roofline": {"bound": "hbm", "achieved": round_gbs, "peak": peak, "unit": "GB/s",

@@ -679,7 +679,10 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
 
 // Merges the split-KV partials the kernel above left behind: one CTA per (work item, kv head), and only the CTA of a
 // split request's first chunk has work -- it combines that (request, head)'s chunks in chunk order (deterministic) and
-// writes the normalised rows.  Thread = one 4-dim column of one row at a time.
+// writes the normalised rows.  Thread = one 4-dim column of one row at a time; blockIdx.y shares a (request, head)'s
+// elements out over kMergeSlices CTAs, because a thread's elements are strictly one after another (two dependent passes
+// over the chunks each) and the kernel is bound by that latency, not by its few megabytes.
+constexpr int kMergeSlices = 3;
 __global__ void __launch_bounds__(128)
 verify_attn_umma_merge_kernel(const __grid_constant__ AttnLaunch a) {
     const int Hkv = a.shape.Hkv, Hq = a.shape.Hq, G = Hq / Hkv, MS = a.m_stride;
@@ -690,7 +693,7 @@ verify_attn_umma_merge_kernel(const __grid_constant__ AttnLaunch a) {
     const int64_t slot0 = (int64_t)it.part_base * Hkv + head;                 // chunk c sits at slot0 + c * Hkv
     const int64_t row_base = it.row0;
     const int M = G * (it.gamma + 1);
-    for (int e = threadIdx.x; e < M * 32; e += 128) {
+    for (int e = blockIdx.y * 128 + threadIdx.x; e < M * 32; e += 128 * kMergeSlices) {
         const int m = e >> 5, d4 = e & 31;
         float mstar = -INFINITY;
         for (int c = 0; c < nch; ++c) mstar = fmaxf(mstar, __ldcg(a.part_ml + ((slot0 + (int64_t)c * Hkv) * MS + m) * 2));
@@ -741,7 +744,7 @@ cudaError_t launch_attn_umma(const AttnLaunch& a, cudaStream_t stream, int n_sms
     verify_attn_umma_kernel<<<grid, kThreads, kSmemBytes, stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || !a.any_split) return e;
-    verify_attn_umma_merge_kernel<<<(unsigned)n_units, 128, 0, stream>>>(a);
+    verify_attn_umma_merge_kernel<<<dim3((unsigned)n_units, kMergeSlices), 128, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

@@ -39,6 +39,15 @@ def test_many_units_per_cta_and_layers():
     base._check(o, res)
 
 
+@pytest.mark.parametrize("chunk_blocks", [24, 40, 0])
+def test_many_units_of_several_tiles_per_cta(chunk_blocks):
+    """Units of three, five and more 128-key tiles, about ten units per persistent CTA: the tile streams change
+    parity from unit to unit, and the unit that a stream writes out changes with them."""
+    cfg = base._cfg("ulong", batch=40, gamma=8, ctx=("uniform", 500, 2600), seed=175)
+    _, _, o, lse, res = base._run(cfg, chunk_blocks=chunk_blocks, want_lse=True)
+    base._check(o, res, lse)
+
+
 def test_fused_round_and_poisoned_tail_slots():
     rnd._run_round(rnd.MULTI, 2)
     rnd._run_round(rnd.ALLMIG, 3)
