@@ -129,6 +129,10 @@ enum {
                                              the reassigned ones are still being copied ...                    */
     NSD_FLAG_ROUND_SPLIT_NEVER = 1 << 5,  /* ... or never (default: only when the copy is long enough to be
                                              worth a second launch)                                            */
+    NSD_FLAG_NO_DEPENDENT_LAUNCH = 1 << 6, /* nsd_verify_round: every kernel starts only when the one before it on
+                                             the stream has completed (default: the round's kernels are launched
+                                             as programmatic dependents, so that one sets itself up beside the
+                                             tail of the one before)                                           */
     NSD_FLAG_TEST_STARVE_GATHER = 1 << 30 /* test hook for the bounded waits: the gather arms every barrier with
                                              16 bytes more than its copy delivers, so each wait runs out after
                                              wait_budget polls and nsd_get_status returns NSD_ERR_TIMEOUT; the

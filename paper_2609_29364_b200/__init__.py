@@ -20,5 +20,6 @@ from .api import (  # noqa: F401
     NSD_FLAG_LOGITS_DIRECT,
     NSD_FLAG_ROUND_SPLIT_ALWAYS,
     NSD_FLAG_ROUND_SPLIT_NEVER,
+    NSD_FLAG_NO_DEPENDENT_LAUNCH,
     NSD_FLAG_TEST_STARVE_GATHER,
 )

@@ -38,6 +38,7 @@ NSD_FLAG_ATTN_NO_TCGEN05 = 1 << 2
 NSD_FLAG_LOGITS_DIRECT = 1 << 3
 NSD_FLAG_ROUND_SPLIT_ALWAYS = 1 << 4
 NSD_FLAG_ROUND_SPLIT_NEVER = 1 << 5
+NSD_FLAG_NO_DEPENDENT_LAUNCH = 1 << 6
 NSD_FLAG_TEST_STARVE_GATHER = 1 << 30
 
 

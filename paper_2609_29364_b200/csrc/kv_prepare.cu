@@ -55,6 +55,7 @@ gather_blocks_bulk_kernel(uint16_t* __restrict__ slab, int64_t n_pairs, const in
                           uint32_t starve_bytes) {
     extern __shared__ __align__(128) unsigned char bulk_smem[];
     __shared__ __align__(8) uint64_t full_bar[kBulkSlots];
+    pdl_release_dependents();                           // whatever follows on the stream may set itself up meanwhile
     if (threadIdx.x != 0) return;                       // a single thread drives the copy engine
     for (int s = 0; s < kBulkSlots; ++s)
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&full_bar[s])) : "memory");
@@ -133,6 +134,10 @@ append_tokens_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32
                      const int32_t* __restrict__ kv_indices, const uint16_t* __restrict__ k_new,
                      const uint16_t* __restrict__ v_new, const uint8_t* __restrict__ is_migrated, int32_t subset,
                      int32_t* __restrict__ status) {
+    // Everything up to the stores reads the call's own inputs only; the stores go into blocks that the kernel before
+    // this one on the stream (a copy into the same blocks, or the attention of the layer that shares the slab) may
+    // still be writing or reading.
+    pdl_release_dependents();
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t n_rows = (int64_t)batch * (gamma + 1);
@@ -170,6 +175,7 @@ append_tokens_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32
     uint16_t* dstb = slab + (int64_t)b * sh.block_elems() + (int64_t)kv * sh.Hkv * sh.tile_elems() + (int64_t)slot * sh.D;
     const int vec_per_head = sh.D / 8;                              // 16-byte pieces per head vector
     const int n_vec = sh.Hkv * vec_per_head;
+    pdl_wait();
     for (int i = lane; i < n_vec; i += 32) {
         const int h = i / vec_per_head, c = i - h * vec_per_head;
         const int4 v = __ldg(reinterpret_cast<const int4*>(srcv + (int64_t)h * sh.D) + c);
@@ -256,13 +262,12 @@ cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const
 cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int64_t* q_indptr,
                           const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices, const uint16_t* k_new,
                           const uint16_t* v_new, const uint8_t* is_migrated, int32_t subset, int32_t* status,
-                          cudaStream_t stream) {
+                          cudaStream_t stream, bool pdl) {
     const int64_t warps = 2LL * batch * (gamma + 1);
     if (warps <= 0) return cudaSuccess;
     const int grid = (int)((warps * 32 + 255) / 256);
-    append_tokens_kernel<<<grid, 256, 0, stream>>>(slab, s, batch, gamma, q_indptr, ctx_len, kv_indptr, kv_indices, k_new, v_new,
-                                                   is_migrated, subset, status);
-    return cudaGetLastError();
+    return launch_kernel(append_tokens_kernel, dim3(grid), dim3(256), 0, stream, pdl, slab, s, batch, gamma, q_indptr, ctx_len,
+                         kv_indptr, kv_indices, k_new, v_new, is_migrated, subset, status);
 }
 
 cudaError_t launch_commit(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int64_t* q_indptr,

@@ -62,6 +62,7 @@ struct nsd_ctx {
     std::vector<const void*> tmap_slab;
     std::vector<char> tmap3_ok;
     int n_sms;
+    bool pdl;                  // nsd_verify_round launches its kernels as programmatic dependents of one another
     int round_split;           // first layer of a round with reassigned requests: 0 = by size, 1 = always attend resident and reassigned requests separately, 2 = never
     int logits_feed;           // acceptance from logits: 1 = rows through the shared-memory ring where aligned (default), 0 = direct loads
     int attn_feed_tma;         // mma.sync kernel: K/V tiles by tensor copies where that is the faster feed (default), 0 = cp.async everywhere
@@ -266,6 +267,7 @@ static nsd_status create_impl(const nsd_config* cfg, void* d_workspace, size_t w
     ctx->attn_tcgen05 = (cfg->flags & NSD_FLAG_ATTN_NO_TCGEN05) ? 0 : ((cfg->flags & NSD_FLAG_ATTN_TCGEN05) ? 2 : 1);
     ctx->round_split = (cfg->flags & NSD_FLAG_ROUND_SPLIT_ALWAYS) ? 1 : ((cfg->flags & NSD_FLAG_ROUND_SPLIT_NEVER) ? 2 : 0);
     ctx->logits_feed = (cfg->flags & NSD_FLAG_LOGITS_DIRECT) ? 0 : 1;
+    ctx->pdl = !(cfg->flags & NSD_FLAG_NO_DEPENDENT_LAUNCH);
     ctx->wait_budget = cfg->wait_budget > 0 ? (uint32_t)cfg->wait_budget : 0u;
     ctx->starve_gather = (cfg->flags & NSD_FLAG_TEST_STARVE_GATHER) ? 16u : 0u;
     *out = ctx;
@@ -534,7 +536,8 @@ struct FuseArgs {
 
 nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* o, float* lse, int32_t gamma,
                         const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices, int32_t layer,
-                        int32_t subset, cudaStream_t st, const FuseArgs* fuse = nullptr) {
+                        int32_t subset, cudaStream_t st, const FuseArgs* fuse = nullptr, bool pdl = false) {
+    // pdl: the first launch follows a kernel of the same call on the stream and may be launched as its programmatic dependent
     AttnLaunch a{};
     if (fuse) {
         a.fuse = 1;
@@ -589,8 +592,11 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
         if (a.tmap_valid && ctx->attn_tcgen05 && attn_umma_supported(a) && (ctx->attn_tcgen05 == 2 || attn_umma_preferred(a))) {
             NSD_CUDA(ctx, launch_attn_umma(a, st, ctx->n_sms));
             ctx->launches += a.any_split ? 2 : 1;                            // the engine's merge kernel follows when a request is split
+            pdl = ctx->pdl;                                                  // what comes next follows a kernel of this call
             continue;
         }
+        a.pdl = pdl;
+        pdl = ctx->pdl;
         NSD_CUDA(ctx, launch_attn(a, st));
         ctx->launches++;
     }
@@ -702,10 +708,21 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
     // on the resident list, and attending that list before the copy event would read blocks still being written.
     const bool can_split = ctx->plan_has_mig && ctx->n_mig_items > 0 && ctx->plan_src_blocks == n_pairs;
     const bool split_first = can_split && (ctx->round_split == 1 || (ctx->round_split == 0 && copy_bytes >= (384LL << 20)));
-    if (overlap) {
+    // A first layer that waits for its copy anyway runs the copy on the caller's stream: no event hop.
+    const bool first_copy_inline = overlap && !split_first;
+    if (overlap && (L > 1 || !first_copy_inline)) {
         NSD_CUDA(ctx, cudaEventRecord(ctx->ev_start, st));
         NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_start, 0));
     }
+    // Kernels of this round that follow a kernel of this round on the caller's stream are launched as its programmatic
+    // dependents: each reads its own inputs and sets itself up beside the tail of the one before, and waits
+    // (griddepcontrol.wait) before it touches the pool or writes an output.
+    bool chained = false;
+    auto dep = [&]() {
+        const bool d = ctx->pdl && chained;
+        chained = true;
+        return d;
+    };
     for (int l = 0; l < L; ++l) {
         uint16_t* slab = slab_ptr(ctx, a->kv_pool, l);
         if (hook) NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_in[l], 0));
@@ -715,28 +732,34 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
             // spare slabs -- and the copy of layer l + 1 is under way while layer l attends: Run || Prepare, layer by
             // layer.  The new tokens' rows, which a model only has once it reaches the layer, are appended on the
             // main stream, for every request, right before the layer's attention.
-            if (l >= S) NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_attn[l - S], 0));
-            NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, a->mig_src, a->mig_dst, ctx->d_status, ctx->n_sms, ctx->wait_budget, ctx->starve_gather, ctx->side));
-            NSD_CUDA(ctx, cudaEventRecord(ctx->ev_prep[l], ctx->side));
+            const bool copy_inline = l == 0 && first_copy_inline;
+            if (copy_inline) {
+                NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, a->mig_src, a->mig_dst, ctx->d_status, ctx->n_sms, ctx->wait_budget, ctx->starve_gather, st));
+                chained = true;
+            } else {
+                if (l >= S) NSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_attn[l - S], 0));
+                NSD_CUDA(ctx, launch_gather(ctx->shape, slab, n_pairs, a->mig_src, a->mig_dst, ctx->d_status, ctx->n_sms, ctx->wait_budget, ctx->starve_gather, ctx->side));
+                NSD_CUDA(ctx, cudaEventRecord(ctx->ev_prep[l], ctx->side));
+            }
             ctx->launches++;
             nsd_status s;
             if (l == 0 && split_first) {
                 // nothing to hide the first copy behind but the first layer itself: its resident requests go first
                 NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices, k_new, v_new,
-                                            a->is_migrated, 1, ctx->d_status, st));
-                s = attn_enqueue(ctx, a->kv_pool, q, o, nullptr, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, 0, 1, st);
+                                            a->is_migrated, 1, ctx->d_status, st, dep()));
+                s = attn_enqueue(ctx, a->kv_pool, q, o, nullptr, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, 0, 1, st, nullptr, dep());
                 if (s != NSD_OK) return s;
                 NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_prep[0], 0));
                 NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices, k_new, v_new,
-                                            a->is_migrated, 2, ctx->d_status, st));
-                s = attn_enqueue(ctx, a->kv_pool, q, o, nullptr, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, 0, 2, st);
+                                            a->is_migrated, 2, ctx->d_status, st, dep()));
+                s = attn_enqueue(ctx, a->kv_pool, q, o, nullptr, gamma, a->ctx_len, a->kv_indptr, a->kv_indices, 0, 2, st, nullptr, dep());
                 ctx->launches += 2;
             } else {
-                NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_prep[l], 0));
+                if (!copy_inline) NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_prep[l], 0));
                 NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices,
-                                            k_new + l * kv_layer, v_new + l * kv_layer, nullptr, 0, ctx->d_status, st));
+                                            k_new + l * kv_layer, v_new + l * kv_layer, nullptr, 0, ctx->d_status, st, dep()));
                 s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
-                                 a->kv_indptr, a->kv_indices, l, 0, st);
+                                 a->kv_indptr, a->kv_indices, l, 0, st, nullptr, dep());
                 ctx->launches++;
             }
             if (s != NSD_OK) return s;
@@ -745,18 +768,18 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
             // gather-through: only the resident requests are appended by the copy kernels; attention itself
             // moves the reassigned requests' blocks and new tokens while it streams them
             NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices,
-                                        k_new + l * kv_layer, v_new + l * kv_layer, a->is_migrated, 1, ctx->d_status, st));
+                                        k_new + l * kv_layer, v_new + l * kv_layer, a->is_migrated, 1, ctx->d_status, st, dep()));
             ctx->launches++;
             const FuseArgs f{a->mig_src, k_new + l * kv_layer, v_new + l * kv_layer};
             nsd_status s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
-                                        a->kv_indptr, a->kv_indices, l, 0, st, &f);
+                                        a->kv_indptr, a->kv_indices, l, 0, st, &f, dep());
             if (s != NSD_OK) return s;
         } else {
             NSD_CUDA(ctx, launch_append(ctx->shape, slab, batch, gamma, qi, a->ctx_len, a->kv_indptr, a->kv_indices,
-                                        k_new + l * kv_layer, v_new + l * kv_layer, nullptr, 0, ctx->d_status, st));
+                                        k_new + l * kv_layer, v_new + l * kv_layer, nullptr, 0, ctx->d_status, st, dep()));
             ctx->launches++;
             nsd_status s = attn_enqueue(ctx, a->kv_pool, q + l * q_layer, o + l * q_layer, nullptr, gamma, a->ctx_len,
-                                        a->kv_indptr, a->kv_indices, l, 0, st);
+                                        a->kv_indptr, a->kv_indices, l, 0, st, nullptr, dep());
             if (s != NSD_OK) return s;
         }
         if (hook) {
@@ -771,7 +794,8 @@ nsd_status round_impl(nsd_ctx* ctx, const nsd_round_args* a, void* stream, const
         NSD_CUDA(ctx, cudaStreamWaitEvent(st, hook->inputs_ready, 0));
     }
     NSD_CUDA(ctx, launch_accept(a->p, a->q_draft, a->draft_tok, a->u_acc, a->u_smp, batch, gamma, ctx->cfg.vocab_size, qi,
-                                a->ctx_len, a->acc_len, a->out_tok, a->new_ctx_len, ctx->d_status, ctx->accept_split, st));
+                                a->ctx_len, a->acc_len, a->out_tok, a->new_ctx_len, ctx->d_status, ctx->accept_split, st,
+                                hook ? false : dep()));
     ctx->launches++;
     if (hook) NSD_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_down_done, 0));      // the caller's stream covers the read-back
     return NSD_OK;

@@ -8,6 +8,32 @@
 
 namespace nsd {
 
+// ---- programmatic dependent launch -------------------------------------------------------------
+// A kernel launched with `pdl` may become resident while the kernel before it on the stream is still running (as
+// soon as every CTA of that one has let its dependents go, or has exited).  It may read its own inputs and set
+// itself up, and must execute pdl_wait() before it touches anything the predecessor writes, or writes anything the
+// predecessor still reads; the wait returns when the predecessor grid has completed and its writes are visible.
+// Without the attribute both instructions do nothing, so one kernel serves both kinds of launch.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... P, typename... A>
+inline cudaError_t launch_kernel(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl, A... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+#endif
+
 // One unit of attention work: a range of KV blocks of one request.  The grid
 // runs one CTA per (item, kv head).
 struct __align__(16) AttnItem {
@@ -66,6 +92,7 @@ struct AttnLaunch {
     uint32_t wait_budget;        // polls per bounded barrier wait, 0 = the kernel's default
     int32_t tmap3_valid;         // tmap3 describes pool_slab
     int32_t any_split;           // some request of the plan has more than one chunk (the tcgen05 engine then launches its merge)
+    int32_t pdl;                 // host side only: launch as a programmatic dependent of the kernel before it on the stream
     CUtensorMap tmap;
     CUtensorMap tmap3;           // tcgen05 engine: 3-D view whose box is a block's whole [16 keys][128 dims] tile
 };
@@ -78,7 +105,7 @@ cudaError_t launch_gather(const Shape& s, uint16_t* slab, int64_t n_pairs, const
 cudaError_t launch_append(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int64_t* q_indptr,
                           const int32_t* ctx_len, const int64_t* kv_indptr, const int32_t* kv_indices, const uint16_t* k_new,
                           const uint16_t* v_new, const uint8_t* is_migrated, int32_t subset, int32_t* status,
-                          cudaStream_t stream);
+                          cudaStream_t stream, bool pdl = false);
 cudaError_t launch_commit(const Shape& s, uint16_t* slab, int32_t batch, int32_t gamma, const int64_t* q_indptr,
                           const int32_t* ctx_len, const int32_t* acc_len, const int64_t* kv_indptr, const int32_t* kv_indices,
                           const int64_t* exp_indptr, const int32_t* exp_indices, int32_t* new_ctx_len, int32_t* status,
@@ -102,7 +129,7 @@ struct AcceptSplit {
 cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
                           const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int64_t* q_indptr,
                           const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
-                          const AcceptSplit& split, cudaStream_t stream);
+                          const AcceptSplit& split, cudaStream_t stream, bool pdl = false);
 
 cudaError_t launch_accept_logits(const void* logits, int32_t logits_bf16, float temperature, const float* q,
                                  const int32_t* draft_tok, const float* u_acc, const float* u_smp, int32_t batch,

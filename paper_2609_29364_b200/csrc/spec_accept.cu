@@ -111,6 +111,7 @@ __device__ __forceinline__ void spec_accept_body(const AcceptArgs& a) {
         d0 = row0 - r;
         gamma = (int)(a.q_indptr[r + 1] - row0) - 1;
         if (gamma < 0 || gamma > a.gamma) {      // an impossible depth: reported, nothing of the request is read
+            pdl_wait();
             if (tid == 0 && part == 0) {
                 atomicOr(a.status, STATUS_BAD_TOKEN);
                 atomicCAS(a.status + 1, 0, r + 1);
@@ -148,6 +149,9 @@ __device__ __forceinline__ void spec_accept_body(const AcceptArgs& a) {
         if (lane == 0) s_n = m ? (__ffs(m) - 1) : gamma;
     }
     __syncthreads();
+    // The tests above read the call's own inputs; the sweep and every output wait for the kernel before this one on
+    // the stream (in a round: the last layer's attention, beside whose tail the tests ran).
+    pdl_wait();
     const int n = s_n;
     const float* prow = p_req + (int64_t)n * vocab;
     const float* qrow = q_req + (int64_t)(n < gamma ? n : 0) * vocab;   // unused when n == gamma
@@ -331,7 +335,7 @@ __global__ void __launch_bounds__(kAcceptThreads) spec_accept_split_kernel(const
 cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_tok, const float* u_acc,
                           const float* u_smp, int32_t batch, int32_t gamma, int32_t vocab, const int64_t* q_indptr,
                           const int32_t* ctx_len, int32_t* acc_len, int32_t* out_tok, int32_t* new_ctx_len, int32_t* status,
-                          const AcceptSplit& sp, cudaStream_t stream) {
+                          const AcceptSplit& sp, cudaStream_t stream, bool pdl) {
     if (batch <= 0) return cudaSuccess;
     const int n_seg = (vocab + kSeg - 1) / kSeg;
     const size_t smem = (size_t)(n_seg + 1) * sizeof(double);
@@ -350,9 +354,8 @@ cudaError_t launch_accept(const float* p, const float* q, const int32_t* draft_t
     }
     const AcceptArgs a{p, q, draft_tok, u_acc, u_smp, gamma, vocab, q_indptr, ctx_len, acc_len, out_tok, new_ctx_len, status,
                        split, sp.scratch, sp.counters};
-    if (split == 1) spec_accept_kernel<<<batch, kAcceptThreads, smem, stream>>>(a);
-    else spec_accept_split_kernel<<<batch * split, kAcceptThreads, smem, stream>>>(a);
-    return cudaGetLastError();
+    if (split == 1) return launch_kernel(spec_accept_kernel, dim3(batch), dim3(kAcceptThreads), smem, stream, pdl, a);
+    return launch_kernel(spec_accept_split_kernel, dim3(batch * split), dim3(kAcceptThreads), smem, stream, pdl, a);
 }
 
 }  // namespace nsd

@@ -172,6 +172,7 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     constexpr int TILE = Tile<D, TK>::kBytes;
     constexpr int ROWS_PAD = NW * NTW * 8;        // query rows incl. padding
     using SM = Smem<D, TK, kStages, ROWS_PAD, TMA>;
+    pdl_release_dependents();                     // the next kernel on the stream may set itself up beside this grid's last wave
     constexpr int STAGE = SM::kStageBytes;
     constexpr int OPITCH = SM::kOutPitch;
     constexpr int ROWS_PER_STEP = NT / CPR;       // rows one pass of all threads covers in a block copy
@@ -311,6 +312,9 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
         cp_async_commit();
     };
 
+    // Up to here the CTA has read its own inputs only (work item, block table) and set up shared memory; from here on it
+    // reads the pool, which the kernel before this one on the stream (the append, a copy) writes.
+    pdl_wait();
 #pragma unroll
     for (int s = 0; s < kStages - 1; ++s) issue_tile(s, s);
 
@@ -719,8 +723,8 @@ verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
 template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false, bool FUSE = false>
 cudaError_t launch_one(const AttnLaunch& a, cudaStream_t stream) {
     const int64_t grid = (int64_t)a.n_items * a.shape.Hkv;
-    verify_attn_kernel<D, NW, NTW, TK, kStages, TMA, FUSE><<<(unsigned)grid, NW * 32, Smem<D, TK, kStages, NW * NTW * 8, TMA>::kBytes, stream>>>(a);
-    return cudaGetLastError();
+    return launch_kernel(verify_attn_kernel<D, NW, NTW, TK, kStages, TMA, FUSE>, dim3((unsigned)grid), dim3(NW * 32),
+                         Smem<D, TK, kStages, NW * NTW * 8, TMA>::kBytes, stream, a.pdl != 0, a);
 }
 
 template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false, bool FUSE = false>
