@@ -20,7 +20,9 @@
 //               first 64, warps 4, 5 the rest; warp w reaches TMEM lanes 32 (w & 3) .. +31).  Read the
 //               scores, mask, half-tile maximum, exchange it with the row's other warp, running maximum
 //               (refreshed only when a score outgrows it by 2^8: then the row of O is rescaled in TMEM,
-//               rare), P = 2^(s - m) as bf16 over the first 64 columns of the same S buffer.
+//               rare), P = 2^(s - m) as bf16 over the first 64 columns of the same S buffer.  From a
+//               unit's second tile on P is formed with the maximum as it stands while the exchange is
+//               under way, and formed again in the rare case that the exchange moves the maximum.
 //   warps 2-3 / 10-11  K producers / V producers, each pair into its own ring of 32 KiB stages, each warp bringing
 //               half of every tile (one warp's copies top out near 40 GB/s).  A K tile is sixteen
 //               TMA boxes of 16 keys x 64 dims (the 128-byte swizzle caps a box row at 64 dims, and the
@@ -192,6 +194,21 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
           "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr));
+}
+// 16 columns, for the rare paths that must not cost the common one its registers
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
@@ -491,6 +508,7 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
         const float sc = rsqrtf(128.f) * kLog2e;
         const int m_row = q * 32 + lane;
         uint32_t g = 0, uidx = 0;
+        uint32_t pair_n = 0;                                // meetings of the row's two warps so far (one per tile, rarely two)
         bool fail = false;                                  // warp-uniform: a wait gave up (the CTA is aborting)
         for (int64_t u = blockIdx.x; u < n_units && !fail; u += gridDim.x, ++uidx) {
             const Unit w = load_unit(a, u);
@@ -510,41 +528,67 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
                 if (fail) break;
                 tc_fence_after();
                 uint32_t sr[64];
-                tmem_ld32(tmem_sb + col0, sr);
-                tmem_ld32(tmem_sb + col0 + 32, sr + 32);
-                tmem_wait_ld();
                 const int key0 = w.item.blk_begin * kBlockSizeU + t * kTileKeys + (int)col0;
                 const int n_vis = vis_stop - key0;          // visible keys of this half tile for this row (may be <= 0 or >= 64)
-                float mx0 = -INFINITY, mx1 = -INFINITY;
                 const bool masked = __any_sync(0xffffffffu, n_vis < 64);
-                // Lanes past M hold no row: they take part in the tensor-memory loads and stores (which are warp-wide) but sit
-                // out the arithmetic, so a warp with few rows costs few lanes' worth of energy.
-                if (live) {
-                    if (masked) {
+                // this half's scores: tensor memory -> registers, hidden keys replaced
+                auto load_scores = [&]() {
+                    tmem_ld32(tmem_sb + col0, sr);
+                    tmem_ld32(tmem_sb + col0 + 32, sr + 32);
+                    tmem_wait_ld();
+                    // Lanes past M hold no row: they take part in the tensor-memory loads and stores (which are warp-wide) but
+                    // sit out the arithmetic, so a warp with few rows costs few lanes' worth of energy.
+                    if (live && masked) {
                         // keys past the chunk (zero-filled boxes) belong to nobody, keys past ctx + i are hidden from row i,
                         // and slots past the last token may hold anything: all replaced by -inf with a select
 #pragma unroll
                         for (int j = 0; j < 64; ++j) sr[j] = j < n_vis ? sr[j] : 0xff800000u;
                     }
+                };
+                // P = 2^(s * sc - m), bf16 pairs, over the scores in place: the 64 keys become 32 words
+                float l0 = 0.f, l1 = 0.f;
+                auto weights = [&]() {
+                    const float nm = m_run == -INFINITY ? 0.f : -m_run;
+                    l0 = 0.f, l1 = 0.f;
+                    if (live) {
+#pragma unroll
+                        for (int j = 0; j < 64; j += 2) {
+                            const float p0 = ex2_approx(fmaf(__uint_as_float(sr[j]), sc, nm));
+                            const float p1 = ex2_approx(fmaf(__uint_as_float(sr[j + 1]), sc, nm));
+                            l0 += p0;
+                            l1 += p1;
+                            sr[j >> 1] = pack_bf16(p0, p1);
+                        }
+                    }
+                };
+                load_scores();
+                float mx0 = -INFINITY, mx1 = -INFINITY;
+                if (live) {
 #pragma unroll
                     for (int j = 0; j < 64; j += 2) {
                         mx0 = fmaxf(mx0, __uint_as_float(sr[j]));
                         mx1 = fmaxf(mx1, __uint_as_float(sr[j + 1]));
                     }
                 }
-                // ---- both halves' maxima: mine out, rendezvous (which also tells the other warp that my scores are in
-                //      registers, so it may write its P over them), the other's in
-                float* xm = xmax_s + (g & 1) * (2 * kRowsMax);
+                // ---- both halves' maxima: mine out, and an arrival that also tells the row's other warp that my scores are
+                //      in registers.  The running maximum moves rarely (only when a score outgrows it by 2^8), so from a
+                //      unit's second tile on the weights are formed with the maximum as it stands while the other half's
+                //      arrival is on its way, and formed again in the rare case that the exchange does move the maximum.
+                float* xm = xmax_s + (pair_n & 1) * (2 * kRowsMax);
                 const float mine = fmaxf(mx0, mx1);
                 xm[(is_b ? kRowsMax : 0) + m_row] = mine;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&pair_bar[q]));
-                if (!mbar_wait(smem_u32(&pair_bar[q]), g & 1, &abort_s, wait_limit)) fail = true;
+                const bool ahead = t > 0;
+                if (ahead) weights();
+                if (!mbar_wait(smem_u32(&pair_bar[q]), pair_n & 1, &abort_s, wait_limit)) fail = true;
                 fail = __any_sync(0xffffffffu, fail);
                 if (fail) break;
+                ++pair_n;
                 const float m_tile = fmaxf(mine, xm[(is_b ? 0 : kRowsMax) + m_row]) * sc;   // -inf when the row sees nothing of this tile
                 const bool outgrown = live && m_tile > m_run + kMaxSlack;      // also the first visible key (m_run = -inf)
-                if (__any_sync(0xffffffffu, outgrown)) {
+                const bool moved = __any_sync(0xffffffffu, outgrown);          // the same answer in both warps of the rows: same rows, same numbers
+                if (moved) {
                     const float m_new = outgrown ? m_tile : m_run;
                     // m_run = -inf: nothing accumulated yet, the factor is irrelevant but must not be NaN
                     const float resc = (outgrown && m_run != -INFINITY) ? ex2_approx(m_run - m_new) : (outgrown ? 0.f : 1.f);
@@ -556,32 +600,34 @@ verify_attn_umma_kernel(const __grid_constant__ AttnLaunch a) {
                         if (fail) break;
                         tc_fence_after();
                         const uint32_t tmem_ob = tmem_o + lane_base + col0;
-#pragma unroll
-                        for (int c = 0; c < 2; ++c) {
-                            uint32_t x[32];
-                            tmem_ld32(tmem_ob + c * 32, x);
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t x[16];
+                            tmem_ld16(tmem_ob + c * 16, x);
                             tmem_wait_ld();
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) x[j] = __float_as_uint(__uint_as_float(x[j]) * resc);
-                            tmem_st32(tmem_ob + c * 32, x);
+                            for (int j = 0; j < 16; ++j) x[j] = __float_as_uint(__uint_as_float(x[j]) * resc);
+                            tmem_st16(tmem_ob + c * 16, x);
                         }
                         tmem_wait_st();
                     }
                     l_run *= resc;
                     m_run = m_new;
                 }
-                // ---- P = 2^(s * sc - m), bf16 pairs: this half's 64 keys become 32 columns among the first 64 of the S buffer
-                const float nm = m_run == -INFINITY ? 0.f : -m_run;
-                float l0 = 0.f, l1 = 0.f;
-                if (live) {
-#pragma unroll
-                    for (int j = 0; j < 64; j += 2) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(sr[j]), sc, nm));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(sr[j + 1]), sc, nm));
-                        l0 += p0;
-                        l1 += p1;
-                        sr[j >> 1] = pack_bf16(p0, p1);
+                if (moved || !ahead) {
+                    if (ahead) {
+                        // the weights formed ahead are void: the scores again (nobody has written P over them yet: a warp
+                        // stores after this point only), and a second meeting so that the other warp's P, which lands on
+                        // columns this warp's scores occupy, waits for this load
+                        load_scores();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&pair_bar[q]));
+                        if (!mbar_wait(smem_u32(&pair_bar[q]), pair_n & 1, &abort_s, wait_limit)) fail = true;
+                        fail = __any_sync(0xffffffffu, fail);
+                        if (fail) break;
+                        ++pair_n;
                     }
+                    weights();
                 }
                 l_run += l0 + l1;
                 tmem_st32(tmem_sb + (col0 >> 1), sr);

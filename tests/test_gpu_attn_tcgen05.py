@@ -48,6 +48,11 @@ def test_many_units_of_several_tiles_per_cta(chunk_blocks):
     base._check(o, res, lse)
 
 
+@pytest.mark.parametrize("gamma", [4, 8, 15])
+def test_running_maximum_moves_late_and_often(gamma):
+    base.test_running_maximum_moves_late_and_often(gamma)
+
+
 def test_fused_round_and_poisoned_tail_slots():
     rnd._run_round(rnd.MULTI, 2)
     rnd._run_round(rnd.ALLMIG, 3)

@@ -17,10 +17,12 @@ def _cfg(name, batch, gamma, ctx, hq=32, hkv=8, d=128, layers=1, frac=0.3, seed=
                          head_dim=d, block_size=16, vocab=100, ctx_dist=ctx, frac_reassigned=frac, seed=seed)
 
 
-def _run(cfg, slabs=None, chunk_blocks=0, subset_pair=False, want_lse=False):
+def _run(cfg, slabs=None, chunk_blocks=0, subset_pair=False, want_lse=False, pool_edit=None):
     slabs = slabs or cfg.num_layers
     meta = W.make_batch_meta(cfg)
     pool0 = np.stack([W.pool_layer(cfg, meta, s) for s in range(slabs)])
+    if pool_edit is not None:
+        pool_edit(pool0, meta)                                                  # in place, before anybody sees the pool
     k_new, v_new = stack_layers(cfg, meta, "kv")
     q = stack_layers(cfg, meta, "q")
     ctx = make_context(cfg, meta, num_slabs=slabs)
@@ -97,6 +99,32 @@ def test_resident_then_reassigned_subsets_cover_everything():
     cfg = _cfg("subsets", batch=12, gamma=4, ctx=("uniform", 20, 900), layers=2, frac=0.5, seed=74)
     _, _, o, _, res = _run(cfg, subset_pair=True, chunk_blocks=8)
     _check(o, res)
+
+
+def _grow_keys_along_the_context(steps):
+    """Pool edit: the committed K rows of every request are multiplied by a factor that steps up along the context
+    (`steps`: (first position, factor) in increasing order), so the largest score of a row rises by far more than
+    2^8 several times on the way -- inside a tile's first keys, inside its last keys, several tiles in."""
+    def edit(pool0, meta):
+        for r in range(len(meta.ctx_len)):
+            blocks = meta.kv_indices[meta.kv_indptr[r]:meta.kv_indptr[r + 1]]
+            for (p0, f), nxt in zip(steps, list(steps[1:]) + [(1 << 30, 0.0)]):
+                for pos in range(p0, min(nxt[0], int(meta.ctx_len[r]))):
+                    k = pool0[:, blocks[pos // 16], 0, :, pos % 16, :]
+                    pool0[:, blocks[pos // 16], 0, :, pos % 16, :] = W.f32_to_bf16(W.bf16_to_f32(k) * np.float32(f))
+    return edit
+
+
+@pytest.mark.parametrize("gamma", [4, 6, 8, 12])
+def test_running_maximum_moves_late_and_often(gamma):
+    """Both engines refresh a row's running maximum lazily and rescale what they have accumulated when it moves: with
+    keys that grow along the context it moves in the first tile's second half, in a later tile's first and last keys,
+    and again far into a long request, for rows that sit in different chunks of a split request too."""
+    steps = ((70, 8.0), (200, 48.0), (390, 6.0), (640, 200.0), (1500, 3.0), (1700, 900.0))
+    cfg = _cfg(f"late{gamma}", batch=9, gamma=gamma, ctx=("fixed", [50, 75, 130, 210, 400, 650, 1000, 1750, 2100]), frac=0.0, seed=181 + gamma)
+    for chunk_blocks in (0, 16):
+        _, _, o, lse, res = _run(cfg, chunk_blocks=chunk_blocks, want_lse=True, pool_edit=_grow_keys_along_the_context(steps))
+        _check(o, res, lse)
 
 
 def test_qwen3_b64_config():
