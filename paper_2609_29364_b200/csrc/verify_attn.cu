@@ -160,7 +160,7 @@ struct Smem {
 // FUSE (TMA-fed variant only; the cp.async variant decides at run time): compiled with the gather-through path.  A
 // separate instantiation, because carrying the path unused cost the plain kernel 5 % (registers, instruction fetch).
 template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false, bool FUSE = false>
-__global__ void __launch_bounds__(NW * 32)
+__global__ void __launch_bounds__(NW * 32, (NW == 2 && NTW == 2) ? 6 : 1)   // two warps x two tiles: six CTAs per SM, as shared memory allows
 verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     static_assert(!TMA || (D == 128 && TK == 16), "the TMA-fed variant covers head_dim 128 with one pool block per stage");
     constexpr int KG = TK / 16;                   // 16-key groups (= pool blocks) per tile
