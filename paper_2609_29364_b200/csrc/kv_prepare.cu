@@ -136,46 +136,52 @@ append_tokens_kernel(uint16_t* __restrict__ slab, Shape sh, int32_t batch, int32
                      int32_t* __restrict__ status) {
     // Everything up to the stores reads the call's own inputs only; the stores go into blocks that the kernel before
     // this one on the stream (a copy into the same blocks, or the attention of the layer that shares the slab) may
-    // still be writing or reading.
+    // still be writing or reading.  Every thread passes the wait, also those with nothing to store: the grid must not
+    // complete before its predecessor has, because the kernel after this one waits for this grid only.
     pdl_release_dependents();
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t n_rows = (int64_t)batch * (gamma + 1);
-    if (warp >= 2 * n_rows) return;
-    const int kv = (int)(warp & 1);
-    int64_t row = warp >> 1;                                        // (request, token) over the padded grid batch x (gamma + 1)
-    const int r = (int)(row / (gamma + 1));
-    const int t = (int)(row - (int64_t)r * (gamma + 1));
-    if (subset != 0 && (int)(is_migrated[r] != 0) != (subset == 2)) return;
-    if (q_indptr) {                                                 // ragged rows: the request has its own depth and row offset
-        const int64_t r0 = q_indptr[r], n = q_indptr[r + 1] - r0;
-        if (n < 1 || n > gamma + 1) {
-            if (lane == 0 && t == 0 && kv == 0) {
-                atomicOr(status, STATUS_BAD_TOKEN);
+    const uint16_t* srcv = nullptr;
+    uint16_t* dstb = nullptr;
+    [&]() {
+        if (warp >= 2 * n_rows) return;
+        const int kv = (int)(warp & 1);
+        int64_t row = warp >> 1;                                    // (request, token) over the padded grid batch x (gamma + 1)
+        const int r = (int)(row / (gamma + 1));
+        const int t = (int)(row - (int64_t)r * (gamma + 1));
+        if (subset != 0 && (int)(is_migrated[r] != 0) != (subset == 2)) return;
+        if (q_indptr) {                                             // ragged rows: the request has its own depth and row offset
+            const int64_t r0 = q_indptr[r], n = q_indptr[r + 1] - r0;
+            if (n < 1 || n > gamma + 1) {
+                if (lane == 0 && t == 0 && kv == 0) {
+                    atomicOr(status, STATUS_BAD_TOKEN);
+                    atomicCAS(status + 1, 0, r + 1);
+                }
+                return;
+            }
+            if (t >= n) return;
+            row = r0 + t;
+        }
+        const int64_t pos = (int64_t)ctx_len[r] + t;
+        const int64_t entry = kv_indptr[r] + pos / sh.bs;
+        const int slot = (int)(pos % sh.bs);
+        int32_t b = -1;
+        if (ctx_len[r] >= 0 && entry < kv_indptr[r + 1]) b = kv_indices[entry];
+        if ((uint32_t)b >= (uint32_t)sh.num_blocks) {
+            if (lane == 0) {
+                atomicOr(status, STATUS_BAD_BLOCK);
                 atomicCAS(status + 1, 0, r + 1);
             }
             return;
         }
-        if (t >= n) return;
-        row = r0 + t;
-    }
-    const int64_t pos = (int64_t)ctx_len[r] + t;
-    const int64_t entry = kv_indptr[r] + pos / sh.bs;
-    const int slot = (int)(pos % sh.bs);
-    int32_t b = -1;
-    if (ctx_len[r] >= 0 && entry < kv_indptr[r + 1]) b = kv_indices[entry];
-    if ((uint32_t)b >= (uint32_t)sh.num_blocks) {
-        if (lane == 0) {
-            atomicOr(status, STATUS_BAD_BLOCK);
-            atomicCAS(status + 1, 0, r + 1);
-        }
-        return;
-    }
-    const uint16_t* srcv = (kv ? v_new : k_new) + row * sh.Hkv * sh.D;
-    uint16_t* dstb = slab + (int64_t)b * sh.block_elems() + (int64_t)kv * sh.Hkv * sh.tile_elems() + (int64_t)slot * sh.D;
+        srcv = (kv ? v_new : k_new) + row * sh.Hkv * sh.D;
+        dstb = slab + (int64_t)b * sh.block_elems() + (int64_t)kv * sh.Hkv * sh.tile_elems() + (int64_t)slot * sh.D;
+    }();
+    pdl_wait();
+    if (!dstb) return;
     const int vec_per_head = sh.D / 8;                              // 16-byte pieces per head vector
     const int n_vec = sh.Hkv * vec_per_head;
-    pdl_wait();
     for (int i = lane; i < n_vec; i += 32) {
         const int h = i / vec_per_head, c = i - h * vec_per_head;
         const int4 v = __ldg(reinterpret_cast<const int4*>(srcv + (int64_t)h * sh.D) + c);
