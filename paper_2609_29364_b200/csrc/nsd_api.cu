@@ -130,7 +130,7 @@ Layout make_layout(const nsd_config* c) {
 }
 
 nsd_status cuda_fail(nsd_ctx* ctx, cudaError_t e, const char* what) {
-    if (ctx) snprintf(ctx->err, sizeof ctx->err, "%s: %s", what, cudaGetErrorString(e));
+    if (ctx) snprintf(ctx->err, sizeof ctx->err, "%.160s: %.80s", what, cudaGetErrorString(e));   // the call's text may be long: keep both parts
     return NSD_ERR_CUDA;
 }
 #define NSD_CUDA(ctx, call)                                         \
