@@ -54,3 +54,15 @@ def test_binding_refuses_to_run_without_the_library(monkeypatch):
     monkeypatch.setattr(api, "_LIB_PATH", os.path.join(ROOT, "no_such_dir", "libnsd.so"))
     with pytest.raises(ImportError):
         api.load_library()
+
+
+def test_binding_flag_constants_match_the_header():
+    """`nsd_config.flags` bits are spelled twice, in the header and in the binding: they must agree, name by name."""
+    import paper_2609_29364_b200.api as api
+
+    text = open(os.path.join(ROOT, "include", "nsd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    header = {name: 1 << int(shift) for name, shift in re.findall(r"\b(NSD_FLAG_[A-Z0-9_]+)\s*=\s*1\s*<<\s*(\d+)", text)}
+    assert len(header) >= 8
+    binding = {name: getattr(api, name) for name in dir(api) if name.startswith("NSD_FLAG_")}
+    assert binding == header

@@ -119,6 +119,16 @@ def test_multi_layer_round(cfg, slabs, split, monkeypatch):
 
 
 @pytest.mark.parametrize("split", ["always", "never"])
+@pytest.mark.parametrize("cfg,slabs,fuse", [(MULTI, 2, False), (ALLMIG, 1, False), (ALLMIG, 3, True), (MULTI, 5, True)],
+                         ids=["multi_alias2", "allmig_alias1", "allmig_through", "multi_through"])
+def test_round_without_dependent_launches(cfg, slabs, fuse, split, monkeypatch):
+    """The round's kernels are launched as programmatic dependents of one another by default (every other test here);
+    with NSD_FLAG_NO_DEPENDENT_LAUNCH each starts only when the one before it has completed.  Same oracle, same bars."""
+    monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", SPLIT_FLAG[split] | (1 << 6))
+    _run_round(cfg, slabs, fuse=fuse, repeat=2)
+
+
+@pytest.mark.parametrize("split", ["always", "never"])
 def test_round_twice_gives_the_same_state(split, monkeypatch):
     """The round is idempotent on its inputs (what the benchmark relies on)."""
     monkeypatch.setattr(nsd_testlib, "CONTEXT_FLAGS", SPLIT_FLAG[split])
