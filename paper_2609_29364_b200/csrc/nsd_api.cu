@@ -562,6 +562,7 @@ nsd_status attn_enqueue(nsd_ctx* ctx, const void* kv_pool, const void* q, void* 
     a.m_stride = ctx->plan_m_stride;
     a.wait_budget = ctx->wait_budget;
     a.any_split = ctx->plan_split_slots > 0;
+    a.cta_slots = ctx->n_sms * 6;
     const AttnItem* base = subset == 0 ? ctx->d_items_all : (subset == 1 ? ctx->d_items_split : ctx->d_items_split + ctx->n_res);
     const int32_t* grp = subset == 0 ? ctx->grp_all : (subset == 1 ? ctx->grp_res : ctx->grp_mig);
     const int32_t* grp_rows = subset == 0 ? ctx->rows_all : (subset == 1 ? ctx->rows_res : ctx->rows_mig);

@@ -93,6 +93,7 @@ struct AttnLaunch {
     int32_t tmap3_valid;         // tmap3 describes pool_slab
     int32_t any_split;           // some request of the plan has more than one chunk (the tcgen05 engine then launches its merge)
     int32_t pdl;                 // host side only: launch as a programmatic dependent of the kernel before it on the stream
+    int32_t cta_slots;           // host side only: CTAs the machine holds at once (SMs x resident CTAs); 0 = not known
     CUtensorMap tmap;
     CUtensorMap tmap3;           // tcgen05 engine: 3-D view whose box is a block's whole [16 keys][128 dims] tile
 };

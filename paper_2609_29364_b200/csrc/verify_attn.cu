@@ -160,7 +160,7 @@ struct Smem {
 // FUSE (TMA-fed variant only; the cp.async variant decides at run time): compiled with the gather-through path.  A
 // separate instantiation, because carrying the path unused cost the plain kernel 5 % (registers, instruction fetch).
 template <int D, int NW, int NTW, int TK, int kStages, bool TMA = false, bool FUSE = false>
-__global__ void __launch_bounds__(NW * 32, (NW == 2 && NTW == 2) ? 6 : 1)   // two warps x two tiles: six CTAs per SM, as shared memory allows
+__global__ void __launch_bounds__(NW * 32, ((NW == 2 && NTW == 2) || (NW == 3 && NTW == 1)) ? 6 : 1)   // six CTAs per SM, as shared memory allows, also where registers would not
 verify_attn_kernel(const __grid_constant__ AttnLaunch a) {
     static_assert(!TMA || (D == 128 && TK == 16), "the TMA-fed variant covers head_dim 128 with one pool block per stage");
     constexpr int KG = TK / 16;                   // 16-key groups (= pool blocks) per tile
@@ -736,9 +736,11 @@ cudaError_t init_one() {
 // One pool block per stage and a deeper ring gave the most resident warps per SM at the same bytes in flight.
 constexpr int kTileKeys = 16, kStagesD64 = 4, kStagesD128 = 4;
 
-// Row tiles of 8: 1..8 of them, spread over warps of at most three tiles each.
+// Row tiles of 8: 1..8 of them, spread over warps of at most three tiles each; and two or three tiles over as many
+// warps of one tile each, for grids that do not fill the machine.
 #define NSD_ATTN_SHAPES(X, DD, SS) \
-    X(DD, 1, 1, kTileKeys, SS) X(DD, 1, 2, kTileKeys, SS) X(DD, 1, 3, kTileKeys, SS) X(DD, 2, 2, kTileKeys, SS) X(DD, 2, 3, kTileKeys, SS) X(DD, 3, 3, kTileKeys, SS)
+    X(DD, 1, 1, kTileKeys, SS) X(DD, 1, 2, kTileKeys, SS) X(DD, 1, 3, kTileKeys, SS) X(DD, 2, 2, kTileKeys, SS) X(DD, 2, 3, kTileKeys, SS) X(DD, 3, 3, kTileKeys, SS) \
+    X(DD, 2, 1, kTileKeys, SS) X(DD, 3, 1, kTileKeys, SS)
 
 }  // namespace
 
@@ -761,11 +763,14 @@ cudaError_t launch_attn(const AttnLaunch& a, cudaStream_t stream) {
     if (a.n_items <= 0) return cudaSuccess;
     const int nt8 = (a.m_rows + 7) / 8;                  // row tiles needed
     if (nt8 < 1 || nt8 > 8) return cudaErrorInvalidValue;
-    const int nw = (nt8 + 2) / 3, ntw = (nt8 + nw - 1) / nw;
+    int nw = (nt8 + 2) / 3, ntw = (nt8 + nw - 1) / nw;
+    // A grid that fits the machine's CTA slots runs as one wave, and the wave lasts as long as one warp takes over its
+    // longest item's tiles: HBM is not the limit there.  Two or three row tiles then go to as many warps of one tile.
+    if (nw == 1 && ntw > 1 && a.cta_slots > 0 && (int64_t)a.n_items * a.shape.Hkv <= a.cta_slots) nw = ntw, ntw = 1;
     // K/V tiles by tensor copies where that measured faster: the shapes that are bound by HBM (up to 32 stacked rows:
     // +4-6 % at 20-24 rows, +3 % at 28-32).  The five- and six-row-tile shapes are bound by the tensor pipe and by
     // shared-memory reads and ran 8-25 % slower fed this way, so they stay on cp.async.
-    if (a.tma_feed && a.tmap_valid && a.shape.D == 128 && (nw == 1 || (nw == 2 && ntw == 2))) {
+    if (a.tma_feed && a.tmap_valid && a.shape.D == 128 && (nw == 1 || ntw == 1 || (nw == 2 && ntw == 2))) {
 #define NSD_TMA_CASE(DD, WW, TT, KK, SS) \
         if (nw == WW && ntw == TT) return a.fuse ? launch_one<DD, WW, TT, KK, SS, true, true>(a, stream) : launch_one<DD, WW, TT, KK, SS, true>(a, stream);
         NSD_ATTN_SHAPES(NSD_TMA_CASE, 128, kStagesD128)
